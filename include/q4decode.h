@@ -1,0 +1,269 @@
+/*
+ * q4decode — C ABI of the B200 decode-step library.
+ *
+ * One call, q4d_decode_step, is the body of the generation loop of the paper's
+ * continuous-batching scheduler (Algorithm 1): for every request r of the
+ * active batch B it computes token_r = GenerateToken(r, KVCache[r]).  Requests
+ * join and leave B only between steps (Algorithm 1, "admit new requests at
+ * token boundaries" / "remove completed requests immediately"), which is what
+ * q4d_request_admit / q4d_request_release express.  Models are 4-bit quantised
+ * (Section 4, "Setup"); the forward pass is the pre-norm decoder of the model
+ * families of Table 1.
+ *
+ * Conventions
+ *  - Every function returns 0 (Q4D_OK) or a negative Q4D_ERR_* code; a failed
+ *    call changes no state.  q4d_last_error() gives the message of the calling
+ *    thread's last failure.
+ *  - "device" pointers are CUDA device memory owned by the caller and must
+ *    outlive the object they are given to; "host" pointers are ordinary host
+ *    memory read before the call returns.  The library allocates no device
+ *    memory; q4d_model_create allocates pinned host staging and events.  It
+ *    never frees memory it was given.
+ *  - Work is enqueued on the given CUDA stream (a cudaStream_t passed as
+ *    void*; NULL = the default stream) and is asynchronous unless stated.
+ *  - bf16 values are passed as uint16_t bit patterns.
+ *
+ * 4-bit tensor format (a projection with K input and N output features):
+ *    q      uint32 [N][K/8]   element k of a row sits in word k>>3, bits 4*(k&7)..+3
+ *    scales bf16   [N][K/64]  one per group of 64 consecutive input features
+ *    biases bf16   [N][K/64]
+ *    w[j][k] = fl32(scales[j][k/64] * q[j][k] + biases[j][k/64])   (never rounded to bf16)
+ *  K must be a multiple of 256.
+ *
+ * KV pool layout (bf16): [layer][0=K,1=V][block][kv_head][slot 0..15][128];
+ * one block id names the same block in every layer.  Keys are stored after
+ * the rotary embedding.
+ */
+#ifndef Q4DECODE_H
+#define Q4DECODE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define Q4D_OK 0
+#define Q4D_ERR_INVALID_ARG (-1)
+#define Q4D_ERR_UNKNOWN_REQUEST (-2)
+#define Q4D_ERR_DUPLICATE_REQUEST (-3)
+#define Q4D_ERR_BATCH_TOO_LARGE (-4)
+#define Q4D_ERR_BLOCK_TABLE_TOO_SHORT (-5)
+#define Q4D_ERR_BLOCK_OUT_OF_RANGE (-6)
+#define Q4D_ERR_POSITION_OVERFLOW (-7)
+#define Q4D_ERR_WORKSPACE_TOO_SMALL (-8)
+#define Q4D_ERR_CUDA (-9)
+#define Q4D_ERR_TIMEOUT (-10)
+#define Q4D_ERR_UNSUPPORTED (-11)
+
+#define Q4D_MAX_BATCH 16
+#define Q4D_BLOCK_SIZE 16
+#define Q4D_HEAD_DIM 128
+
+/* Shape of the model (plain data). */
+typedef struct {
+  int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim; /* head_dim must be 128 */
+  int32_t mlp_inter, vocab;
+  int32_t group_size /* 64 */, bits /* 4 */;
+  int32_t qk_norm /* 0|1: per-head RMSNorm of q and k before the rotary embedding */;
+  int32_t tie_embeddings /* informational: embed and lm_head may alias */;
+  float rms_eps;
+  int32_t n_experts /* 0 = dense MLP */, top_k, expert_inter, norm_topk_prob;
+  int32_t max_batch /* <= 16 */, max_positions /* rows of the rotary table */;
+} q4d_shape;
+
+/* One 4-bit tensor: three device pointers (format above). */
+typedef struct {
+  const uint32_t* q;
+  const uint16_t* scales;
+  const uint16_t* biases;
+} q4d_qtensor;
+
+/* Per-layer device pointers.  Norm weights are bf16 vectors. */
+typedef struct {
+  const uint16_t *attn_norm, *mlp_norm; /* [hidden] */
+  const uint16_t *q_norm, *k_norm;      /* [128], NULL unless qk_norm */
+  q4d_qtensor wqkv;      /* [(nq+2nkv)*128][hidden], rows: q heads, k heads, v heads */
+  q4d_qtensor wo;        /* [hidden][nq*128] */
+  q4d_qtensor w_gate_up; /* [2*mlp_inter][hidden], rows: gate then up (dense only) */
+  q4d_qtensor w_down;    /* [hidden][mlp_inter] (dense only) */
+  const uint16_t* router;      /* bf16 [n_experts][hidden] (MoE only) */
+  q4d_qtensor experts_gate_up; /* [n_experts][2*expert_inter][hidden] stacked (MoE only) */
+  q4d_qtensor experts_down;    /* [n_experts][hidden][expert_inter] stacked (MoE only) */
+} q4d_layer_weights;
+
+typedef struct {
+  const q4d_layer_weights* layers; /* host array of n_layers entries (copied by model_create) */
+  const uint16_t* final_norm;      /* bf16 [hidden] */
+  q4d_qtensor embed;               /* [vocab][hidden] */
+  q4d_qtensor lm_head;             /* [vocab][hidden] */
+  const float* rope_cos_sin;       /* f32 [max_positions][64][2] = (cos, sin) of position * frequency_i */
+} q4d_weights;
+
+typedef struct q4d_model q4d_model;
+typedef struct q4d_kv_pool q4d_kv_pool;
+
+const char* q4d_last_error(void);
+
+/* ---- model -------------------------------------------------------------- */
+
+/* Bytes of device workspace q4d_model_create needs for this shape (activations,
+ * split-K and split-KV partial sums, per-step metadata).  0 if the shape is
+ * not supported. */
+size_t q4d_model_workspace_bytes(const q4d_shape* shape);
+
+/* Binds a shape to its weights ("model_create(shape config, device weight
+ * pointers)").  `weights` is a host struct of device pointers; the per-layer
+ * array is copied, the tensors are not.  `workspace` is device memory of at
+ * least q4d_model_workspace_bytes(shape), 256-byte aligned, used exclusively by
+ * this model until it is destroyed.  Errors: INVALID_ARG (NULL pointer,
+ * missing tensor), UNSUPPORTED (head_dim != 128, group_size != 64, bits != 4,
+ * widths not multiples of 256, more than 16 q heads per kv head, max_batch
+ * > 16), WORKSPACE_TOO_SMALL, CUDA. */
+int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* workspace,
+                     size_t workspace_bytes, q4d_model** out);
+int q4d_model_destroy(q4d_model* model);
+
+/* ---- paged KV pool and batch membership ------------------------------- */
+
+size_t q4d_kv_pool_bytes(const q4d_shape* shape, int32_t num_blocks, int32_t block_size);
+
+/* Wraps caller-owned device memory (layout in the file header) as the block
+ * pool of `model` ("kv_pool_create(blocks, block_size)").  block_size must be
+ * 16.  The caller allocates blocks to requests and fills prefilled KV; the
+ * library only reads the blocks named in block tables and appends one token
+ * per step. */
+int q4d_kv_pool_create(q4d_model* model, int32_t num_blocks, int32_t block_size, void* pool_mem,
+                       size_t pool_bytes, q4d_kv_pool** out);
+int q4d_kv_pool_destroy(q4d_kv_pool* pool);
+
+/* A request joins the batch between steps (Algorithm 1, admission loop).  Its
+ * first `prefilled_len` tokens already have K, V in the caller's blocks.
+ * Errors: DUPLICATE_REQUEST, POSITION_OVERFLOW (prefilled_len < 0 or
+ * >= max_positions). */
+int q4d_request_admit(q4d_kv_pool* pool, int64_t request_id, int32_t prefilled_len);
+/* A request leaves the batch between steps (Algorithm 1, removal loop). */
+int q4d_request_release(q4d_kv_pool* pool, int64_t request_id);
+/* Tokens cached so far for a request. */
+int q4d_request_len(q4d_kv_pool* pool, int64_t request_id, int32_t* len_out);
+/* Number of admitted requests. */
+int q4d_request_count(q4d_kv_pool* pool, int32_t* count_out);
+
+/* ---- the decode step ---------------------------------------------------- */
+
+/* One token for each of the n listed requests (Algorithm 1, generation loop:
+ * token_r = GenerateToken(r, KVCache[r]) for each r in B).
+ *   request_ids   host  [n]   distinct, all admitted
+ *   last_tokens   host  [n]   the token each request feeds in (0 <= t < vocab)
+ *   block_tables  host  [n][max_blocks]  physical block of tokens 16*i..16*i+15;
+ *                 row r must cover len_r + 1 tokens; the block receiving the
+ *                 new token must not be shared with another request
+ *   next_tokens   device [n]  greedy token (argmax of the logits, lowest index on ties)
+ *   logits        device [n][vocab] f32, or NULL
+ * Outputs are in the order of request_ids.  On success each listed request's
+ * length grows by one; n = 0 is a no-op.  The call validates everything on
+ * the host first (UNKNOWN_REQUEST, DUPLICATE_REQUEST, BATCH_TOO_LARGE,
+ * BLOCK_TABLE_TOO_SHORT, BLOCK_OUT_OF_RANGE, POSITION_OVERFLOW, INVALID_ARG),
+ * then enqueues the kernels and returns without synchronising. */
+int q4d_decode_step(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
+                    const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
+                    int32_t* next_tokens, float* logits, void* cuda_stream);
+
+/* Same step, but the fed-in tokens are read from device memory when the
+ * kernels run (e.g. the next_tokens buffer of the previous step), so a loop
+ * of steps needs no host round trip.  Token values are then not validated on
+ * the host; out-of-range values are clamped into the vocabulary. */
+int q4d_decode_step_chained(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
+                            const int32_t* last_tokens_device, const int32_t* block_tables,
+                            int32_t max_blocks, int32_t* next_tokens, float* logits,
+                            void* cuda_stream);
+
+/* Same step with host outputs: next_tokens_host [n] and, if not NULL,
+ * logits_host [n][vocab] are filled and the stream is synchronised before the
+ * call returns. */
+int q4d_decode_step_host(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
+                         const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
+                         int32_t* next_tokens_host, float* logits_host, void* cuda_stream);
+
+/* ---- instrumentation ---------------------------------------------------- */
+
+/* Kernel classes timed by the profile mode. */
+enum {
+  Q4D_K_EMBED = 0, Q4D_K_RMSNORM, Q4D_K_GEMM_QKV, Q4D_K_ROPE_APPEND, Q4D_K_ATTENTION,
+  Q4D_K_ATTN_MERGE, Q4D_K_GEMM_O, Q4D_K_GEMM_GATE_UP, Q4D_K_GEMM_DOWN, Q4D_K_MOE_ROUTER,
+  Q4D_K_MOE_GATE_UP, Q4D_K_MOE_DOWN, Q4D_K_LM_HEAD, Q4D_K_ARGMAX, Q4D_K_COUNT
+};
+/* With profiling on, every kernel launch of a step is bracketed by CUDA events
+ * on the step's stream.  q4d_profile_read synchronises, adds up the elapsed
+ * milliseconds and launches per class since the last read into ms[Q4D_K_COUNT]
+ * and launches[Q4D_K_COUNT] (host arrays), and clears the record. */
+int q4d_profile_enable(q4d_model* model, int32_t on);
+int q4d_profile_read(q4d_model* model, float* ms, int32_t* launches);
+/* Kernel launches enqueued by this model since creation. */
+int64_t q4d_launch_count(q4d_model* model);
+/* Bytes the most recent step copied host -> device (per-step metadata: tokens,
+ * lengths, block tables, attention work list) and device -> host (only the
+ * host-output variant copies anything back). */
+int q4d_step_io_bytes(q4d_model* model, int64_t* h2d_bytes, int64_t* d2h_bytes);
+
+/* ---- single operations (the kernels of the step, callable alone) -------- */
+/* All pointers are device memory; n <= 16.  `scratch` is device memory of at
+ * least q4d_op_scratch_bytes() bytes, zero-initialised once by the caller and
+ * owned by one stream at a time. */
+size_t q4d_op_scratch_bytes(void);
+
+/* y[r][j] = sum_k w[j][k] x[r][k] with w dequantised on the fly.
+ *   prologue 0: x is bf16 [n][K] (row stride x_stride elements)
+ *   prologue 1: x is bf16 [n][2K] = gate | up; the operand is bf16(silu(gate) * up)
+ *   epilogue 0: out bf16 [n][N] = bf16(y)
+ *   epilogue 1: out bf16 [n][N] updated in place: out = bf16(out + bf16(y))   (residual)
+ *   epilogue 2: out f32  [n][N] = y
+ * out_stride is the element distance between requests in out. */
+int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, int32_t x_stride,
+                int32_t n, int32_t prologue, int32_t epilogue, void* out, int32_t out_stride,
+                void* scratch, void* cuda_stream);
+
+/* y = bf16(x * rsqrt(mean(x^2) + eps) * w), rows of length H. */
+int q4d_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int32_t n, int32_t H, uint16_t* y,
+                void* cuda_stream);
+
+/* x[r] = bf16(dequantised row tokens[r] of the table). */
+int q4d_embed(const q4d_qtensor* table, int32_t vocab, int32_t H, const int32_t* tokens, int32_t n,
+              uint16_t* x, void* cuda_stream);
+
+/* Per-head RMSNorm (if q_norm/k_norm given) and rotary embedding of q and k at
+ * position lens[r]; q goes to q_out bf16 [n][nq][128]; k and v are appended to
+ * the pool at token slot lens[r].  qkv is bf16 [n][(nq+2nkv)*128]. */
+int q4d_rope_append(const uint16_t* qkv, const uint16_t* q_norm, const uint16_t* k_norm, float eps,
+                    const float* rope_cos_sin, int32_t n, int32_t nq, int32_t nkv, const int32_t* lens,
+                    const int32_t* block_tables, int32_t max_blocks, uint16_t* pool_layer_k,
+                    uint16_t* pool_layer_v, uint16_t* q_out, void* cuda_stream);
+
+/* Decode attention of q bf16 [n][nq][128] over tokens 0..lens[r] of each
+ * request in one layer of the pool (split over the KV length, partial results
+ * merged by log-sum-exp).  The lengths are given twice: the host copy plans
+ * the split, the device copy is read by the kernels.  out bf16 [n][nq][128].
+ * The call synchronises the stream before it returns. */
+int q4d_paged_attention(const uint16_t* q, const uint16_t* pool_layer_k, const uint16_t* pool_layer_v,
+                        int32_t n, int32_t nq, int32_t nkv, const int32_t* lens_host,
+                        const int32_t* lens_device, const int32_t* block_tables_device,
+                        int32_t max_blocks, int32_t chunk_tokens /* 0 = auto */, uint16_t* out,
+                        void* scratch, void* cuda_stream);
+
+/* next[r] = argmax_j logits[r][j], lowest index on ties. */
+int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, void* cuda_stream);
+
+/* ---- parity exports ----------------------------------------------------- */
+
+/* out f32 [N][K] = the dequantised weights (bit-exact definition above). */
+int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out_device, void* cuda_stream);
+/* Tokens 0..len-1 of one layer of the pool, gathered through a device block
+ * table into k_out, v_out bf16 [len][n_kv_heads][128]. */
+int q4d_debug_kv_gather(q4d_kv_pool* pool, int32_t layer, const int32_t* block_table_device,
+                        int32_t len, uint16_t* k_out, uint16_t* v_out, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Q4DECODE_H */

@@ -1,0 +1,679 @@
+// C ABI of the q4decode library: objects, host-side validation, and the
+// stream-ordered launch sequence of one decode step.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <string>
+#include <unordered_map>
+#include <unordered_set>
+#include <vector>
+
+#include "../../include/q4decode.h"
+#include "kernels.h"
+
+using namespace q4d;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_last_error = buf;
+  return code;
+}
+
+int fail_cuda(cudaError_t e, const char* what) {
+  return fail(Q4D_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+// Per-step metadata, one contiguous block: header, attention work list, block tables.
+struct MetaLayout {
+  int max_blocks_cap, max_work;
+  size_t off_tokens, off_lens, off_slot_base, off_nchunks, off_bt, off_work, bytes;
+  void init(int max_positions) {
+    max_blocks_cap = (max_positions + kBlockSize - 1) / kBlockSize;
+    max_work = attention_max_work(kMaxBatch, max_positions);
+    size_t o = 0;
+    off_tokens = o, o += kMaxBatch * 4;
+    off_lens = o, o += kMaxBatch * 4;
+    off_slot_base = o, o += kMaxBatch * 4;
+    off_nchunks = o, o += kMaxBatch * 4;
+    off_work = o, o += (size_t)max_work * sizeof(int4);
+    off_bt = o, o += (size_t)kMaxBatch * max_blocks_cap * 4;
+    bytes = align_up(o);
+  }
+};
+
+struct Workspace {
+  size_t x, y, qkv, qbuf, attn, gu, logits, next, gemm_partial, gemm_partial_bytes, counters, part_acc, part_ml,
+      meta, bytes;
+  int counters_len;
+};
+
+bool shape_supported(const q4d_shape& s, std::string* why) {
+  auto bad = [&](const char* m) {
+    if (why) *why = m;
+    return false;
+  };
+  if (s.n_layers < 1 || s.hidden < 256 || s.n_q_heads < 1 || s.n_kv_heads < 1 || s.vocab < 1)
+    return bad("non-positive dimension");
+  if (s.head_dim != kHeadDim) return bad("head_dim must be 128");
+  if (s.group_size != 64 || s.bits != 4) return bad("only 4-bit group-64 weights are supported");
+  if (s.n_q_heads % s.n_kv_heads || s.n_q_heads / s.n_kv_heads > 16) return bad("q heads per kv head must be 1..16");
+  if (s.hidden % 256 || (s.n_q_heads * s.head_dim) % 256) return bad("hidden and nq*128 must be multiples of 256");
+  if (s.max_batch < 1 || s.max_batch > kMaxBatch) return bad("max_batch must be 1..16");
+  if (s.max_positions < 1) return bad("max_positions must be positive");
+  if (s.n_experts == 0) {
+    if (s.mlp_inter < 256 || s.mlp_inter % 256) return bad("mlp_inter must be a positive multiple of 256");
+  } else {
+    return bad("MoE layers are not supported yet");
+  }
+  return true;
+}
+
+Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
+  Workspace w;
+  size_t o = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o += align_up(bytes);
+    return at;
+  };
+  const size_t B = kMaxBatch;
+  const int nqkv = (s.n_q_heads + 2 * s.n_kv_heads) * kHeadDim;
+  w.x = take(B * s.hidden * 2);
+  w.y = take(B * s.hidden * 2);
+  w.qkv = take(B * nqkv * 2);
+  w.qbuf = take(B * s.n_q_heads * kHeadDim * 2);
+  w.attn = take(B * s.n_q_heads * kHeadDim * 2);
+  w.gu = take(B * 2 * (size_t)s.mlp_inter * 2);
+  w.logits = take(B * (size_t)s.vocab * 4);
+  w.next = take(B * 4);
+  size_t pb = 0;
+  int cl = 0;
+  auto gemm = [&](int N, int K) {
+    pb = std::max(pb, gemm_partial_bytes(N, K));
+    cl = std::max(cl, gemm_counters_needed(N));
+  };
+  gemm(nqkv, s.hidden);
+  gemm(s.hidden, s.n_q_heads * kHeadDim);
+  gemm(2 * s.mlp_inter, s.hidden);
+  gemm(s.hidden, s.mlp_inter);
+  gemm(s.vocab, s.hidden);
+  w.gemm_partial_bytes = pb;
+  w.gemm_partial = take(pb);
+  w.counters_len = cl;
+  w.counters = take((size_t)cl * 4);
+  w.part_acc = take((size_t)ml.max_work * s.n_q_heads * kHeadDim * 4);
+  w.part_ml = take((size_t)ml.max_work * s.n_q_heads * 2 * 4);
+  w.meta = take(ml.bytes);
+  w.bytes = o;
+  return w;
+}
+
+constexpr int kStagingSlots = 8;
+
+struct ProfileRec {
+  cudaEvent_t a, b;
+  int cls;
+};
+
+}  // namespace
+
+struct q4d_model {
+  q4d_shape sh;
+  std::vector<q4d_layer_weights> layers;
+  q4d_weights w;
+  unsigned char* ws;
+  Workspace lay;
+  MetaLayout ml;
+  int sm_count;
+  // pinned staging ring for the per-step metadata
+  unsigned char* staging[kStagingSlots];
+  cudaEvent_t staging_done[kStagingSlots];
+  bool staging_used[kStagingSlots];
+  int staging_next;
+  // instrumentation
+  bool profile;
+  std::vector<ProfileRec> prof_recs;
+  std::vector<cudaEvent_t> prof_free;
+  int64_t launches;
+  int64_t last_h2d, last_d2h;
+  int32_t* host_next;  // pinned, for the host-output variant
+};
+
+struct q4d_kv_pool {
+  q4d_model* model;
+  int32_t num_blocks;
+  uint16_t* mem;
+  std::unordered_map<int64_t, int32_t> lens;
+};
+
+namespace {
+
+template <typename T>
+T* at(q4d_model* m, size_t off) {
+  return reinterpret_cast<T*>(m->ws + off);
+}
+
+// Runs one launch, bracketed by events in profile mode.
+template <typename F>
+cudaError_t timed(q4d_model* m, int cls, cudaStream_t s, F&& f) {
+  ProfileRec rec{nullptr, nullptr, cls};
+  if (m->profile) {
+    for (cudaEvent_t* ev : {&rec.a, &rec.b}) {
+      if (!m->prof_free.empty()) {
+        *ev = m->prof_free.back();
+        m->prof_free.pop_back();
+      } else {
+        cudaError_t e = cudaEventCreate(ev);
+        if (e != cudaSuccess) return e;
+      }
+    }
+    cudaEventRecord(rec.a, s);
+  }
+  cudaError_t e = f();
+  m->launches++;
+  if (m->profile) {
+    cudaEventRecord(rec.b, s);
+    m->prof_recs.push_back(rec);
+  }
+  return e;
+}
+
+GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint16_t* x, int x_stride, int n, int pro,
+                   int epi, void* out, int out_stride) {
+  GemmArgs a;
+  a.qw = t.q, a.scales = t.scales, a.biases = t.biases;
+  a.N = N, a.K = K, a.x = x, a.x_stride = x_stride, a.n = n, a.prologue = pro, a.epilogue = epi;
+  a.out = out, a.out_stride = out_stride;
+  a.partial = at<float>(m, m->lay.gemm_partial), a.partial_bytes = m->lay.gemm_partial_bytes;
+  a.counters = at<int>(m, m->lay.counters), a.counters_len = m->lay.counters_len;
+  return a;
+}
+
+bool qt_ok(const q4d_qtensor& t) { return t.q && t.scales && t.biases; }
+
+int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* tokens_host,
+              const int32_t* tokens_dev, const int32_t* bt, int32_t max_blocks, int32_t* next_dev, float* logits_dev,
+              cudaStream_t s) {
+  if (!m || !pool || pool->model != m) return fail(Q4D_ERR_INVALID_ARG, "decode_step: model/pool mismatch or NULL");
+  if (n < 0) return fail(Q4D_ERR_INVALID_ARG, "decode_step: n < 0");
+  if (n == 0) return Q4D_OK;
+  if (n > m->sh.max_batch)
+    return fail(Q4D_ERR_BATCH_TOO_LARGE, "decode_step: n = %d exceeds max_batch %d", n, m->sh.max_batch);
+  if (!ids || (!tokens_host && !tokens_dev) || !bt || !next_dev || max_blocks < 1)
+    return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL argument");
+  const q4d_shape& sh = m->sh;
+
+  // ---- validate on the host; nothing is changed before this block passes ----
+  int32_t lens[kMaxBatch];
+  {
+    std::unordered_set<int64_t> seen;
+    for (int r = 0; r < n; ++r) {
+      const long long id = (long long)ids[r];
+      if (!seen.insert(ids[r]).second)
+        return fail(Q4D_ERR_DUPLICATE_REQUEST, "decode_step: request %lld listed twice", id);
+      auto it = pool->lens.find(ids[r]);
+      if (it == pool->lens.end())
+        return fail(Q4D_ERR_UNKNOWN_REQUEST, "decode_step: request %lld was not admitted", id);
+      lens[r] = it->second;
+      if (lens[r] + 1 > sh.max_positions)
+        return fail(Q4D_ERR_POSITION_OVERFLOW, "decode_step: request %lld is at max_positions", id);
+      const int need = (lens[r] + 1 + kBlockSize - 1) / kBlockSize;
+      if (need > max_blocks)
+        return fail(Q4D_ERR_BLOCK_TABLE_TOO_SHORT, "decode_step: request %lld needs %d blocks, table has %d", id, need,
+                    max_blocks);
+      for (int i = 0; i < need; ++i) {
+        const int b = bt[(size_t)r * max_blocks + i];
+        if (b < 0 || b >= pool->num_blocks)
+          return fail(Q4D_ERR_BLOCK_OUT_OF_RANGE, "decode_step: request %lld block %d = %d outside the pool", id, i, b);
+      }
+      if (tokens_host && (tokens_host[r] < 0 || tokens_host[r] >= sh.vocab))
+        return fail(Q4D_ERR_INVALID_ARG, "decode_step: token %d outside the vocabulary", tokens_host[r]);
+    }
+  }
+
+  // ---- per-step metadata: stage in pinned memory, copy to the device ----
+  const MetaLayout& ml = m->ml;
+  const int slot = m->staging_next;
+  m->staging_next = (slot + 1) % kStagingSlots;
+  if (m->staging_used[slot]) {
+    cudaError_t e = cudaEventSynchronize(m->staging_done[slot]);
+    if (e != cudaSuccess) return fail_cuda(e, "staging wait");
+  }
+  unsigned char* st = m->staging[slot];
+  int32_t* h_tokens = reinterpret_cast<int32_t*>(st + ml.off_tokens);
+  int32_t* h_lens = reinterpret_cast<int32_t*>(st + ml.off_lens);
+  int32_t* h_slot = reinterpret_cast<int32_t*>(st + ml.off_slot_base);
+  int32_t* h_nch = reinterpret_cast<int32_t*>(st + ml.off_nchunks);
+  int4* h_work = reinterpret_cast<int4*>(st + ml.off_work);
+  int32_t* h_bt = reinterpret_cast<int32_t*>(st + ml.off_bt);
+  for (int r = 0; r < n; ++r) {
+    h_tokens[r] = tokens_host ? tokens_host[r] : 0;
+    h_lens[r] = lens[r];
+    const int need = (lens[r] + 1 + kBlockSize - 1) / kBlockSize;  // <= max_blocks_cap since len < max_positions
+    for (int i = 0; i < ml.max_blocks_cap; ++i)
+      h_bt[(size_t)r * ml.max_blocks_cap + i] = i < need ? bt[(size_t)r * max_blocks + i] : 0;
+  }
+  const AttnPlan plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
+  unsigned char* dmeta = m->ws + m->lay.meta;
+  const size_t head_bytes = ml.off_work + (size_t)plan.n_work * sizeof(int4);
+  const size_t bt_bytes = (size_t)n * ml.max_blocks_cap * 4;
+  cudaError_t e = cudaMemcpyAsync(dmeta, st, head_bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dmeta + ml.off_bt, st + ml.off_bt, bt_bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(e, "metadata copy");
+  cudaEventRecord(m->staging_done[slot], s);
+  m->staging_used[slot] = true;
+  m->last_h2d = (int64_t)(head_bytes + bt_bytes);
+  m->last_d2h = 0;
+
+  const int32_t* d_tokens = tokens_dev ? tokens_dev : reinterpret_cast<const int32_t*>(dmeta + ml.off_tokens);
+  const int32_t* d_lens = reinterpret_cast<const int32_t*>(dmeta + ml.off_lens);
+  const int32_t* d_bt = reinterpret_cast<const int32_t*>(dmeta + ml.off_bt);
+
+  // ---- the launch sequence ----
+  const int H = sh.hidden, nq = sh.n_q_heads, nkv = sh.n_kv_heads, I = sh.mlp_inter, V = sh.vocab;
+  const int nqkv = (nq + 2 * nkv) * kHeadDim;
+  uint16_t* x = at<uint16_t>(m, m->lay.x);
+  uint16_t* y = at<uint16_t>(m, m->lay.y);
+  uint16_t* qkv = at<uint16_t>(m, m->lay.qkv);
+  uint16_t* qbuf = at<uint16_t>(m, m->lay.qbuf);
+  uint16_t* attn = at<uint16_t>(m, m->lay.attn);
+  uint16_t* gu = at<uint16_t>(m, m->lay.gu);
+  float* logits = logits_dev ? logits_dev : at<float>(m, m->lay.logits);
+  const size_t layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
+
+#define Q4D_LAUNCH(cls, expr)                                                 \
+  do {                                                                        \
+    cudaError_t le = timed(m, cls, s, [&]() -> cudaError_t { return expr; }); \
+    if (le != cudaSuccess) return fail_cuda(le, #cls);                        \
+  } while (0)
+
+  Q4D_LAUNCH(Q4D_K_EMBED, launch_embed(m->w.embed.q, m->w.embed.scales, m->w.embed.biases, V, H, d_tokens, n, x, s));
+  for (int l = 0; l < sh.n_layers; ++l) {
+    const q4d_layer_weights& lw = m->layers[l];
+    uint16_t* kpool = pool->mem + (size_t)(2 * l) * layer_elems;
+    uint16_t* vpool = kpool + layer_elems;
+    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, y, s));
+    Q4D_LAUNCH(Q4D_K_GEMM_QKV,
+               launch_q4_gemm(gemm_args(m, lw.wqkv, nqkv, H, y, H, n, PRO_PLAIN, EPI_BF16, qkv, nqkv), s));
+    RopeArgs ra;
+    ra.qkv = qkv, ra.q_norm = sh.qk_norm ? lw.q_norm : nullptr, ra.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
+    ra.eps = sh.rms_eps, ra.rope = m->w.rope_cos_sin, ra.n = n, ra.nq = nq, ra.nkv = nkv, ra.lens = d_lens;
+    ra.block_tables = d_bt, ra.max_blocks = ml.max_blocks_cap, ra.kpool = kpool, ra.vpool = vpool, ra.q_out = qbuf;
+    Q4D_LAUNCH(Q4D_K_ROPE_APPEND, launch_rope_append(ra, s));
+    AttnArgs aa;
+    aa.q = qbuf, aa.kpool = kpool, aa.vpool = vpool, aa.block_tables = d_bt, aa.lens = d_lens;
+    aa.work = reinterpret_cast<const int4*>(dmeta + ml.off_work);
+    aa.slot_base = reinterpret_cast<const int32_t*>(dmeta + ml.off_slot_base);
+    aa.nchunks = reinterpret_cast<const int32_t*>(dmeta + ml.off_nchunks);
+    aa.n_work = plan.n_work, aa.n = n, aa.nq = nq, aa.nkv = nkv, aa.max_blocks = ml.max_blocks_cap;
+    aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml), aa.out = attn;
+    Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
+    Q4D_LAUNCH(Q4D_K_ATTN_MERGE, launch_attention_merge(aa, s));
+    Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, nq * kHeadDim, attn, nq * kHeadDim, n, PRO_PLAIN,
+                                                      EPI_RESIDUAL, x, H), s));
+    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, y, s));
+    Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP,
+               launch_q4_gemm(gemm_args(m, lw.w_gate_up, 2 * I, H, y, H, n, PRO_PLAIN, EPI_BF16, gu, 2 * I), s));
+    Q4D_LAUNCH(Q4D_K_GEMM_DOWN,
+               launch_q4_gemm(gemm_args(m, lw.w_down, H, I, gu, 2 * I, n, PRO_SILU_MUL, EPI_RESIDUAL, x, H), s));
+  }
+  Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, y, s));
+  Q4D_LAUNCH(Q4D_K_LM_HEAD,
+             launch_q4_gemm(gemm_args(m, m->w.lm_head, V, H, y, H, n, PRO_PLAIN, EPI_F32, logits, V), s));
+  Q4D_LAUNCH(Q4D_K_ARGMAX, launch_argmax(logits, n, V, next_dev, s));
+#undef Q4D_LAUNCH
+
+  for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
+  return Q4D_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* q4d_last_error(void) { return g_last_error.c_str(); }
+
+size_t q4d_model_workspace_bytes(const q4d_shape* shape) {
+  std::string why;
+  if (!shape || !shape_supported(*shape, &why)) {
+    fail(Q4D_ERR_UNSUPPORTED, "workspace_bytes: %s", shape ? why.c_str() : "NULL shape");
+    return 0;
+  }
+  MetaLayout ml;
+  ml.init(shape->max_positions);
+  return carve(*shape, ml).bytes;
+}
+
+int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* workspace, size_t workspace_bytes,
+                     q4d_model** out) {
+  if (!shape || !weights || !workspace || !out) return fail(Q4D_ERR_INVALID_ARG, "model_create: NULL argument");
+  std::string why;
+  if (!shape_supported(*shape, &why)) return fail(Q4D_ERR_UNSUPPORTED, "model_create: %s", why.c_str());
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign)
+    return fail(Q4D_ERR_INVALID_ARG, "model_create: workspace must be 256-byte aligned");
+  if (!weights->layers || !weights->final_norm || !weights->rope_cos_sin || !qt_ok(weights->embed) ||
+      !qt_ok(weights->lm_head))
+    return fail(Q4D_ERR_INVALID_ARG, "model_create: missing tensor");
+  for (int l = 0; l < shape->n_layers; ++l) {
+    const q4d_layer_weights& lw = weights->layers[l];
+    if (!lw.attn_norm || !lw.mlp_norm || !qt_ok(lw.wqkv) || !qt_ok(lw.wo) || !qt_ok(lw.w_gate_up) ||
+        !qt_ok(lw.w_down) || (shape->qk_norm && (!lw.q_norm || !lw.k_norm)))
+      return fail(Q4D_ERR_INVALID_ARG, "model_create: layer %d has a missing tensor", l);
+  }
+  MetaLayout ml;
+  ml.init(shape->max_positions);
+  cudaError_t e = gemm_init();
+  if (e == cudaSuccess) e = attention_init();
+  if (e != cudaSuccess) return fail_cuda(e, "kernel init");
+  const Workspace lay = carve(*shape, ml);
+  if (workspace_bytes < lay.bytes)
+    return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "model_create: workspace %zu < %zu", workspace_bytes, lay.bytes);
+  q4d_model* m = new (std::nothrow) q4d_model();
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "model_create: out of host memory");
+  m->sh = *shape;
+  m->layers.assign(weights->layers, weights->layers + shape->n_layers);
+  m->w = *weights;
+  m->w.layers = m->layers.data();
+  m->ws = static_cast<unsigned char*>(workspace);
+  m->lay = lay;
+  m->ml = ml;
+  m->profile = false;
+  m->launches = 0;
+  m->last_h2d = m->last_d2h = 0;
+  m->staging_next = 0;
+  m->host_next = nullptr;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  for (int i = 0; i < kStagingSlots; ++i)
+    m->staging[i] = nullptr, m->staging_done[i] = nullptr, m->staging_used[i] = false;
+  for (int i = 0; i < kStagingSlots && e == cudaSuccess; ++i) {
+    e = cudaMallocHost(reinterpret_cast<void**>(&m->staging[i]), ml.bytes);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->staging_done[i], cudaEventDisableTiming);
+  }
+  if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_next), kMaxBatch * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    q4d_model_destroy(m);
+    return fail_cuda(e, "model_create");
+  }
+  *out = m;
+  return Q4D_OK;
+}
+
+int q4d_model_destroy(q4d_model* m) {
+  if (!m) return Q4D_OK;
+  for (int i = 0; i < kStagingSlots; ++i) {
+    if (m->staging[i]) cudaFreeHost(m->staging[i]);
+    if (m->staging_done[i]) cudaEventDestroy(m->staging_done[i]);
+  }
+  if (m->host_next) cudaFreeHost(m->host_next);
+  for (auto& r : m->prof_recs) cudaEventDestroy(r.a), cudaEventDestroy(r.b);
+  for (auto ev : m->prof_free) cudaEventDestroy(ev);
+  delete m;
+  return Q4D_OK;
+}
+
+size_t q4d_kv_pool_bytes(const q4d_shape* shape, int32_t num_blocks, int32_t block_size) {
+  if (!shape || num_blocks < 1 || block_size != kBlockSize) return 0;
+  return (size_t)shape->n_layers * 2 * num_blocks * shape->n_kv_heads * block_size * shape->head_dim * 2;
+}
+
+int q4d_kv_pool_create(q4d_model* model, int32_t num_blocks, int32_t block_size, void* pool_mem, size_t pool_bytes,
+                       q4d_kv_pool** out) {
+  if (!model || !pool_mem || !out) return fail(Q4D_ERR_INVALID_ARG, "kv_pool_create: NULL argument");
+  if (block_size != kBlockSize) return fail(Q4D_ERR_UNSUPPORTED, "kv_pool_create: block_size must be 16");
+  if (num_blocks < 1) return fail(Q4D_ERR_INVALID_ARG, "kv_pool_create: num_blocks < 1");
+  if (reinterpret_cast<uintptr_t>(pool_mem) % 16)
+    return fail(Q4D_ERR_INVALID_ARG, "kv_pool_create: pool must be 16-byte aligned");
+  const size_t need = q4d_kv_pool_bytes(&model->sh, num_blocks, block_size);
+  if (pool_bytes < need) return fail(Q4D_ERR_INVALID_ARG, "kv_pool_create: pool %zu < %zu bytes", pool_bytes, need);
+  q4d_kv_pool* p = new (std::nothrow) q4d_kv_pool();
+  if (!p) return fail(Q4D_ERR_INVALID_ARG, "kv_pool_create: out of host memory");
+  p->model = model, p->num_blocks = num_blocks, p->mem = static_cast<uint16_t*>(pool_mem);
+  *out = p;
+  return Q4D_OK;
+}
+
+int q4d_kv_pool_destroy(q4d_kv_pool* p) {
+  delete p;
+  return Q4D_OK;
+}
+
+int q4d_request_admit(q4d_kv_pool* p, int64_t id, int32_t prefilled_len) {
+  if (!p) return fail(Q4D_ERR_INVALID_ARG, "request_admit: NULL pool");
+  if (prefilled_len < 0 || prefilled_len >= p->model->sh.max_positions)
+    return fail(Q4D_ERR_POSITION_OVERFLOW, "request_admit: prefilled_len %d outside [0, %d)", prefilled_len,
+                p->model->sh.max_positions);
+  if (p->lens.count(id))
+    return fail(Q4D_ERR_DUPLICATE_REQUEST, "request_admit: request %lld already admitted", (long long)id);
+  p->lens[id] = prefilled_len;
+  return Q4D_OK;
+}
+
+int q4d_request_release(q4d_kv_pool* p, int64_t id) {
+  if (!p) return fail(Q4D_ERR_INVALID_ARG, "request_release: NULL pool");
+  if (!p->lens.erase(id))
+    return fail(Q4D_ERR_UNKNOWN_REQUEST, "request_release: request %lld was not admitted", (long long)id);
+  return Q4D_OK;
+}
+
+int q4d_request_len(q4d_kv_pool* p, int64_t id, int32_t* len_out) {
+  if (!p || !len_out) return fail(Q4D_ERR_INVALID_ARG, "request_len: NULL argument");
+  auto it = p->lens.find(id);
+  if (it == p->lens.end())
+    return fail(Q4D_ERR_UNKNOWN_REQUEST, "request_len: request %lld was not admitted", (long long)id);
+  *len_out = it->second;
+  return Q4D_OK;
+}
+
+int q4d_request_count(q4d_kv_pool* p, int32_t* count_out) {
+  if (!p || !count_out) return fail(Q4D_ERR_INVALID_ARG, "request_count: NULL argument");
+  *count_out = (int32_t)p->lens.size();
+  return Q4D_OK;
+}
+
+int q4d_decode_step(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* last_tokens,
+                    const int32_t* bt, int32_t max_blocks, int32_t* next_tokens, float* logits, void* stream) {
+  if (n > 0 && !last_tokens) return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL last_tokens");
+  return step_impl(m, pool, n, ids, last_tokens, nullptr, bt, max_blocks, next_tokens, logits,
+                   static_cast<cudaStream_t>(stream));
+}
+
+int q4d_decode_step_chained(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids,
+                            const int32_t* last_tokens_device, const int32_t* bt, int32_t max_blocks,
+                            int32_t* next_tokens, float* logits, void* stream) {
+  if (n > 0 && !last_tokens_device) return fail(Q4D_ERR_INVALID_ARG, "decode_step_chained: NULL last_tokens_device");
+  return step_impl(m, pool, n, ids, nullptr, last_tokens_device, bt, max_blocks, next_tokens, logits,
+                   static_cast<cudaStream_t>(stream));
+}
+
+int q4d_decode_step_host(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* last_tokens,
+                         const int32_t* bt, int32_t max_blocks, int32_t* next_tokens_host, float* logits_host,
+                         void* stream) {
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "decode_step_host: NULL model");
+  if (n > 0 && (!last_tokens || !next_tokens_host))
+    return fail(Q4D_ERR_INVALID_ARG, "decode_step_host: NULL argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* d_next = at<int32_t>(m, m->lay.next);
+  float* d_logits = at<float>(m, m->lay.logits);
+  const int rc = step_impl(m, pool, n, ids, last_tokens, nullptr, bt, max_blocks, d_next, d_logits, s);
+  if (rc != Q4D_OK || n == 0) return rc;
+  cudaError_t e = cudaMemcpyAsync(m->host_next, d_next, (size_t)n * 4, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess && logits_host)
+    e = cudaMemcpyAsync(logits_host, d_logits, (size_t)n * m->sh.vocab * 4, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(e, "decode_step_host");
+  memcpy(next_tokens_host, m->host_next, (size_t)n * 4);
+  m->last_d2h = (int64_t)n * 4 + (logits_host ? (int64_t)n * m->sh.vocab * 4 : 0);
+  return Q4D_OK;
+}
+
+int q4d_profile_enable(q4d_model* m, int32_t on) {
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "profile_enable: NULL model");
+  m->profile = on != 0;
+  return Q4D_OK;
+}
+
+int q4d_profile_read(q4d_model* m, float* ms, int32_t* launches) {
+  if (!m || !ms || !launches) return fail(Q4D_ERR_INVALID_ARG, "profile_read: NULL argument");
+  for (int i = 0; i < Q4D_K_COUNT; ++i) ms[i] = 0.0f, launches[i] = 0;
+  for (auto& r : m->prof_recs) {
+    cudaError_t e = cudaEventSynchronize(r.b);
+    float t = 0.0f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&t, r.a, r.b);
+    if (e != cudaSuccess) return fail_cuda(e, "profile_read");
+    ms[r.cls] += t;
+    launches[r.cls] += 1;
+    m->prof_free.push_back(r.a);
+    m->prof_free.push_back(r.b);
+  }
+  m->prof_recs.clear();
+  return Q4D_OK;
+}
+
+int64_t q4d_launch_count(q4d_model* m) { return m ? m->launches : 0; }
+
+int q4d_step_io_bytes(q4d_model* m, int64_t* h2d, int64_t* d2h) {
+  if (!m || !h2d || !d2h) return fail(Q4D_ERR_INVALID_ARG, "step_io_bytes: NULL argument");
+  *h2d = m->last_h2d, *d2h = m->last_d2h;
+  return Q4D_OK;
+}
+
+// ---- single operations ------------------------------------------------------------
+
+namespace {
+constexpr size_t kOpCounters = 64 * 1024;  // bytes
+constexpr size_t kOpGemmPartial = 48ull << 20;
+constexpr size_t kOpAttnMeta = 1ull << 20;
+constexpr size_t kOpPartAcc = 64ull << 20;
+constexpr size_t kOpPartMl = 1ull << 20;
+}  // namespace
+
+size_t q4d_op_scratch_bytes(void) { return kOpCounters + kOpGemmPartial + kOpAttnMeta + kOpPartAcc + kOpPartMl; }
+
+int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, int32_t x_stride, int32_t n,
+                int32_t prologue, int32_t epilogue, void* out, int32_t out_stride, void* scratch, void* stream) {
+  if (!w || !qt_ok(*w) || !x || !out || !scratch) return fail(Q4D_ERR_INVALID_ARG, "q4_gemm: NULL argument");
+  if (n < 0 || n > kMaxBatch || N < 1 || K < 256 || K % 256 || x_stride % 8 || prologue < 0 || prologue > 1 ||
+      epilogue < 0 || epilogue > 2)
+    return fail(Q4D_ERR_INVALID_ARG, "q4_gemm: bad shape (K must be a multiple of 256, n <= 16)");
+  if (gemm_partial_bytes(N, K) > kOpGemmPartial || (size_t)gemm_counters_needed(N) * 4 > kOpCounters)
+    return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "q4_gemm: shape needs more scratch than q4d_op_scratch_bytes provides");
+  GemmArgs a;
+  a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.x = x, a.x_stride = x_stride, a.n = n;
+  a.prologue = prologue, a.epilogue = epilogue, a.out = out, a.out_stride = out_stride;
+  unsigned char* sc = static_cast<unsigned char*>(scratch);
+  a.counters = reinterpret_cast<int*>(sc), a.counters_len = (int)(kOpCounters / 4);
+  a.partial = reinterpret_cast<float*>(sc + kOpCounters), a.partial_bytes = kOpGemmPartial;
+  cudaError_t e = launch_q4_gemm(a, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "q4_gemm");
+}
+
+int q4d_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int32_t n, int32_t H, uint16_t* y, void* stream) {
+  if (!x || !w || !y || n < 0 || H < 2 || H % 2) return fail(Q4D_ERR_INVALID_ARG, "rmsnorm: bad argument");
+  cudaError_t e = launch_rmsnorm(x, w, eps, n, H, y, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "rmsnorm");
+}
+
+int q4d_embed(const q4d_qtensor* t, int32_t vocab, int32_t H, const int32_t* tokens, int32_t n, uint16_t* x,
+              void* stream) {
+  if (!t || !qt_ok(*t) || !tokens || !x || n < 0 || H % 64) return fail(Q4D_ERR_INVALID_ARG, "embed: bad argument");
+  cudaError_t e = launch_embed(t->q, t->scales, t->biases, vocab, H, tokens, n, x, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "embed");
+}
+
+int q4d_rope_append(const uint16_t* qkv, const uint16_t* q_norm, const uint16_t* k_norm, float eps, const float* rope,
+                    int32_t n, int32_t nq, int32_t nkv, const int32_t* lens, const int32_t* bt, int32_t max_blocks,
+                    uint16_t* kpool, uint16_t* vpool, uint16_t* q_out, void* stream) {
+  if (!qkv || !rope || !lens || !bt || !kpool || !vpool || !q_out || n < 0 || nq < 1 || nkv < 1)
+    return fail(Q4D_ERR_INVALID_ARG, "rope_append: bad argument");
+  RopeArgs a;
+  a.qkv = qkv, a.q_norm = q_norm, a.k_norm = k_norm, a.eps = eps, a.rope = rope, a.n = n, a.nq = nq, a.nkv = nkv;
+  a.lens = lens, a.block_tables = bt, a.max_blocks = max_blocks, a.kpool = kpool, a.vpool = vpool, a.q_out = q_out;
+  cudaError_t e = launch_rope_append(a, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "rope_append");
+}
+
+int q4d_paged_attention(const uint16_t* q, const uint16_t* kpool, const uint16_t* vpool, int32_t n, int32_t nq,
+                        int32_t nkv, const int32_t* lens_host, const int32_t* lens_device, const int32_t* bt_device,
+                        int32_t max_blocks, int32_t chunk_tokens, uint16_t* out, void* scratch, void* stream) {
+  if (!q || !kpool || !vpool || !lens_host || !lens_device || !bt_device || !out || !scratch)
+    return fail(Q4D_ERR_INVALID_ARG, "paged_attention: NULL argument");
+  if (n < 0 || n > kMaxBatch || nq < 1 || nkv < 1 || nq % nkv || nq / nkv > 16)
+    return fail(Q4D_ERR_INVALID_ARG, "paged_attention: bad head counts or batch");
+  if (n == 0) return Q4D_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int sms = 148, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const size_t by_meta = (kOpAttnMeta - 1024) / sizeof(int4);
+  const size_t by_acc = kOpPartAcc / ((size_t)nq * kHeadDim * 4), by_ml = kOpPartMl / ((size_t)nq * 8);
+  const int max_work = (int)std::min(by_meta, std::min(by_acc, by_ml));
+  std::vector<int4> work(max_work);
+  int32_t head[2 * kMaxBatch];
+  const AttnPlan plan =
+      plan_attention(lens_host, n, nkv, chunk_tokens, sms, work.data(), head, head + kMaxBatch, max_work);
+  long long want = 0;
+  for (int r = 0; r < n; ++r) want += ((lens_host[r] + 1 + 15) / 16 + plan.chunk_tiles - 1) / plan.chunk_tiles;
+  if (want != plan.n_work)
+    return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "paged_attention: too many chunks for the op scratch");
+  unsigned char* sc = static_cast<unsigned char*>(scratch) + kOpCounters + kOpGemmPartial;
+  cudaError_t e = cudaMemcpyAsync(sc, head, sizeof head, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(sc + 1024, work.data(), (size_t)plan.n_work * sizeof(int4), cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(e, "paged_attention metadata");
+  AttnArgs a;
+  a.q = q, a.kpool = kpool, a.vpool = vpool, a.block_tables = bt_device, a.lens = lens_device;
+  a.work = reinterpret_cast<const int4*>(sc + 1024);
+  a.slot_base = reinterpret_cast<const int32_t*>(sc), a.nchunks = reinterpret_cast<const int32_t*>(sc) + kMaxBatch;
+  a.n_work = plan.n_work, a.n = n, a.nq = nq, a.nkv = nkv, a.max_blocks = max_blocks;
+  a.part_acc = reinterpret_cast<float*>(sc + kOpAttnMeta);
+  a.part_ml = reinterpret_cast<float*>(sc + kOpAttnMeta + kOpPartAcc);
+  a.out = out;
+  e = launch_paged_attention(a, s);
+  if (e == cudaSuccess) e = launch_attention_merge(a, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);  // the host work list must outlive the copy
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "paged_attention");
+}
+
+int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, void* stream) {
+  if (!logits || !next || n < 0 || vocab < 1) return fail(Q4D_ERR_INVALID_ARG, "argmax: bad argument");
+  cudaError_t e = launch_argmax(logits, n, vocab, next, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "argmax");
+}
+
+int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out, void* stream) {
+  if (!w || !qt_ok(*w) || !out || N < 1 || K < 64 || K % 64)
+    return fail(Q4D_ERR_INVALID_ARG, "debug_dequant: bad argument");
+  cudaError_t e = launch_dequant(w->q, w->scales, w->biases, N, K, out, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "debug_dequant");
+}
+
+int q4d_debug_kv_gather(q4d_kv_pool* p, int32_t layer, const int32_t* bt_device, int32_t len, uint16_t* k_out,
+                        uint16_t* v_out, void* stream) {
+  if (!p || !bt_device || !k_out || !v_out || len < 0 || layer < 0 || layer >= p->model->sh.n_layers)
+    return fail(Q4D_ERR_INVALID_ARG, "debug_kv_gather: bad argument");
+  const size_t layer_elems = (size_t)p->num_blocks * p->model->sh.n_kv_heads * kBlockSize * kHeadDim;
+  const uint16_t* kpool = p->mem + (size_t)(2 * layer) * layer_elems;
+  cudaError_t e = launch_kv_gather(kpool, kpool + layer_elems, p->model->sh.n_kv_heads, bt_device, len, k_out, v_out,
+                                   static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "debug_kv_gather");
+}
+
+}  // extern "C"

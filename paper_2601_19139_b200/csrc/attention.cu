@@ -1,0 +1,356 @@
+// GQA decode attention over a paged KV pool, split over the KV length with a
+// log-sum-exp merge, plus the kernel that prepares q and appends k, v.
+//
+// For request r, q head a (kv head h = a / G) and cached tokens t = 0..len_r:
+//   s_t = q_a . k_t / sqrt(128),  P = softmax(s),  out_a = bf16(sum_t P_t v_t)
+//
+// Work item = (request, kv head, chunk of consecutive 16-token blocks).  A CTA
+// of four warps takes one item; each warp walks its share of the chunk's
+// blocks through a private cp.async ring (one stage = the 4 KB K block and the
+// 4 KB V block of that kv head), computes scores for the G query heads of the
+// kv head with m16n8k16 MMAs (rows = query heads, padded to 16), keeps a
+// running (max, sum, accumulator) per head, and multiplies P into V with P
+// split into two bf16 terms so the product keeps ~16 bits of P.  The warps'
+// states are merged in shared memory and written as one partial result per
+// item; a second kernel merges the partial results of a request.
+#include <math.h>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace q4d {
+
+namespace {
+
+constexpr int kAttnThreads = 128;
+constexpr int kAttnWarps = 4;
+constexpr int kAttnStages = 3;
+constexpr int kTileBytes = 16 * 128 * 2;    // one block of one kv head: 16 tokens x 128 x bf16
+constexpr int kAttnStage = 2 * kTileBytes;  // K then V
+constexpr float kScaleLog2 = 0.08838834764831845f * 1.4426950408889634f;  // log2(e) / sqrt(128)
+
+__global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const AttnArgs p) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const int G = p.nq / p.nkv;
+  const int h = blockIdx.y;
+
+  grid_dependency_wait();
+
+  for (int item = blockIdx.x; item < p.n_work; item += gridDim.x) {
+    const int4 w = p.work[item];
+    const int r = w.x, tile_begin = w.y, tile_end = w.z, slot = w.w;
+    const int T = p.lens[r] + 1;
+    const int32_t* bt = p.block_tables + (size_t)r * p.max_blocks;
+    unsigned char* ring = smem + warp * (kAttnStages * kAttnStage);
+
+    // Q fragments: rows = query heads of this kv head (zero beyond G), k = head dimension.
+    uint32_t qa[8][4];
+    {
+      const uint16_t* q0 = p.q + ((size_t)r * p.nq + (size_t)h * G + g) * kHeadDim;
+      const uint16_t* q1 = q0 + 8 * kHeadDim;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t) : 0u;
+        qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t) : 0u;
+        qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t + 8) : 0u;
+        qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t + 8) : 0u;
+      }
+    }
+
+    auto issue_tile = [&](int tile, int stage) {
+      const int blk = bt[tile];
+      const size_t base = ((size_t)blk * p.nkv + h) * (16 * kHeadDim);
+      const unsigned char* ksrc = reinterpret_cast<const unsigned char*>(p.kpool + base);
+      const unsigned char* vsrc = reinterpret_cast<const unsigned char*>(p.vpool + base);
+      unsigned char* dst = ring + stage * kAttnStage;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = i * 32 + lane;  // 16-byte chunk of the 4 KB block
+        const int tok = c >> 4, c16 = c & 15;
+        const int off = tok * 256 + ((c16 ^ (tok & 7)) << 4);
+        cp_async16(dst + off, ksrc + c * 16);
+        cp_async16(dst + kTileBytes + off, vsrc + c * 16);
+      }
+    };
+
+    float o[16][4];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.0f, l_hi = 0.0f;
+
+    const int first = tile_begin + warp;
+    const int my_tiles = (first < tile_end) ? (tile_end - first + kAttnWarps - 1) / kAttnWarps : 0;
+#pragma unroll
+    for (int s = 0; s < kAttnStages - 1; ++s) {
+      if (s < my_tiles) issue_tile(first + s * kAttnWarps, s);
+      cp_async_commit();
+    }
+
+    for (int it = 0; it < my_tiles; ++it) {
+      const int tile = first + it * kAttnWarps;
+      if (it + kAttnStages - 1 < my_tiles)
+        issue_tile(first + (it + kAttnStages - 1) * kAttnWarps, (it + kAttnStages - 1) % kAttnStages);
+      cp_async_commit();
+      cp_async_wait<kAttnStages - 1>();
+      __syncwarp();
+      const unsigned char* sK = ring + (it % kAttnStages) * kAttnStage;
+      const unsigned char* sV = sK + kTileBytes;
+
+      // scores S[head][token] for the 16 tokens of the block
+      float s[2][4];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.0f;
+#pragma unroll
+        for (int kp = 0; kp < 4; ++kp) {
+          uint32_t kb[4];
+          const int tok = 8 * j + (lane & 7), chunk = 4 * kp + (lane >> 3);
+          ldmatrix_x4(kb, sK + tok * 256 + ((chunk ^ (tok & 7)) << 4));
+          mma_bf16(s[j], qa[2 * kp][0], qa[2 * kp][1], qa[2 * kp][2], qa[2 * kp][3], kb[0], kb[1]);
+          mma_bf16(s[j], qa[2 * kp + 1][0], qa[2 * kp + 1][1], qa[2 * kp + 1][2], qa[2 * kp + 1][3], kb[2], kb[3]);
+        }
+      }
+      if (tile * 16 + 16 > T) {  // ragged last block: tokens at or beyond T do not exist
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+            if (tile * 16 + 8 * j + 2 * t + (c & 1) >= T) s[j][c] = -INFINITY;
+      }
+
+      // online softmax, rows g (lo) and g + 8 (hi); m is kept in log2 units
+      float mx_lo = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+      float mx_hi = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+      const float mn_lo = fmaxf(m_lo, mx_lo * kScaleLog2), mn_hi = fmaxf(m_hi, mx_hi * kScaleLog2);
+      const bool grow = (mn_lo > m_lo) || (mn_hi > m_hi);
+      if (__any_sync(0xffffffffu, grow)) {
+        const float c_lo = exp2f(m_lo - mn_lo), c_hi = exp2f(m_hi - mn_hi);
+        l_lo *= c_lo;
+        l_hi *= c_hi;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          o[j][0] *= c_lo, o[j][1] *= c_lo;
+          o[j][2] *= c_hi, o[j][3] *= c_hi;
+        }
+        m_lo = mn_lo, m_hi = mn_hi;
+      }
+      uint32_t ph[4], pl[4];  // A fragments of P: hi and lo bf16 terms
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const float p0 = exp2f(fmaf(s[j][0], kScaleLog2, -m_lo)), p1 = exp2f(fmaf(s[j][1], kScaleLog2, -m_lo));
+        const float p2 = exp2f(fmaf(s[j][2], kScaleLog2, -m_hi)), p3 = exp2f(fmaf(s[j][3], kScaleLog2, -m_hi));
+        l_lo += p0 + p1;
+        l_hi += p2 + p3;
+        const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
+        ph[2 * j] = h01, ph[2 * j + 1] = h23;
+        pl[2 * j] = pack_bf16x2(p0 - bf16_lo(h01), p1 - bf16_hi(h01));
+        pl[2 * j + 1] = pack_bf16x2(p2 - bf16_lo(h23), p3 - bf16_hi(h23));
+      }
+
+      // O[head][d] += P[head][token] V[token][d]
+#pragma unroll
+      for (int jp = 0; jp < 8; ++jp) {
+        uint32_t vb[4];
+        const int i = lane >> 3;
+        const int tok = (i & 1) * 8 + (lane & 7), chunk = 2 * jp + (i >> 1);
+        ldmatrix_x4_trans(vb, sV + tok * 256 + ((chunk ^ (tok & 7)) << 4));
+        mma_bf16(o[2 * jp], ph[0], ph[1], ph[2], ph[3], vb[0], vb[1]);
+        mma_bf16(o[2 * jp], pl[0], pl[1], pl[2], pl[3], vb[0], vb[1]);
+        mma_bf16(o[2 * jp + 1], ph[0], ph[1], ph[2], ph[3], vb[2], vb[3]);
+        mma_bf16(o[2 * jp + 1], pl[0], pl[1], pl[2], pl[3], vb[2], vb[3]);
+      }
+      __syncwarp();
+    }
+    cp_async_wait<0>();
+
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+    // merge the four warps through shared memory (overlays the rings)
+    __syncthreads();
+    float* sO = reinterpret_cast<float*>(smem);   // [warp][16][128]
+    float* sM = sO + kAttnWarps * 16 * kHeadDim;  // [warp][16]
+    float* sL = sM + kAttnWarps * 16;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      float* row_lo = sO + ((warp * 16 + g) * kHeadDim) + 8 * j + 2 * t;
+      *reinterpret_cast<float2*>(row_lo) = make_float2(o[j][0], o[j][1]);
+      *reinterpret_cast<float2*>(row_lo + 8 * kHeadDim) = make_float2(o[j][2], o[j][3]);
+    }
+    if (t == 0) {
+      sM[warp * 16 + g] = m_lo, sM[warp * 16 + g + 8] = m_hi;
+      sL[warp * 16 + g] = l_lo, sL[warp * 16 + g + 8] = l_hi;
+    }
+    __syncthreads();
+    {
+      const int d = threadIdx.x;
+      for (int a = 0; a < G; ++a) {
+        float M = sM[a];
+#pragma unroll
+        for (int ww = 1; ww < kAttnWarps; ++ww) M = fmaxf(M, sM[ww * 16 + a]);
+        float num = 0.0f, den = 0.0f;
+#pragma unroll
+        for (int ww = 0; ww < kAttnWarps; ++ww) {
+          const float e = exp2f(sM[ww * 16 + a] - M);
+          num = fmaf(e, sO[(ww * 16 + a) * kHeadDim + d], num);
+          den = fmaf(e, sL[ww * 16 + a], den);
+        }
+        const size_t qh = (size_t)slot * p.nq + (size_t)h * G + a;
+        p.part_acc[qh * kHeadDim + d] = num;
+        if (d == 0) {
+          p.part_ml[qh * 2] = M;
+          p.part_ml[qh * 2 + 1] = den;
+        }
+      }
+    }
+    __syncthreads();
+  }
+}
+
+// out[r][a] = bf16(sum_c 2^(m_c - M) acc_c / sum_c 2^(m_c - M) l_c) over the request's chunks, in chunk order.
+__global__ void __launch_bounds__(kHeadDim) attention_merge_kernel(const AttnArgs p) {
+  grid_dependency_wait();
+  const int r = blockIdx.x, a = blockIdx.y, d = threadIdx.x;
+  const int s0 = p.slot_base[r], nc = p.nchunks[r];
+  float M = -INFINITY;
+  for (int c = 0; c < nc; ++c) M = fmaxf(M, p.part_ml[((size_t)(s0 + c) * p.nq + a) * 2]);
+  float num = 0.0f, den = 0.0f;
+  for (int c = 0; c < nc; ++c) {
+    const size_t qh = (size_t)(s0 + c) * p.nq + a;
+    const float e = exp2f(p.part_ml[qh * 2] - M);
+    num = fmaf(e, p.part_acc[qh * kHeadDim + d], num);
+    den = fmaf(e, p.part_ml[qh * 2 + 1], den);
+  }
+  p.out[((size_t)r * p.nq + a) * kHeadDim + d] = f32_to_bf16(num / den);
+}
+
+// One warp per (request, head of qkv): optional RMSNorm over the head, rotary embedding at the
+// request's position, then q -> q_out, k and v -> the pool slot of the new token.
+__global__ void __launch_bounds__(128) rope_append_kernel(const RopeArgs p) {
+  grid_dependency_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int heads = p.nq + 2 * p.nkv;
+  const int hd = blockIdx.x * 4 + warp, r = blockIdx.y;
+  if (hd >= heads) return;
+  const uint16_t* src = p.qkv + ((size_t)r * heads + hd) * kHeadDim;
+  const int pos = p.lens[r];
+  // lane holds elements 2*lane, 2*lane+1 and their rotary partners 64 + 2*lane, 64 + 2*lane + 1
+  const uint32_t wa = *reinterpret_cast<const uint32_t*>(src + 2 * lane);
+  const uint32_t wb = *reinterpret_cast<const uint32_t*>(src + 64 + 2 * lane);
+  uint32_t oa = wa, ob = wb;
+  if (hd < p.nq + p.nkv) {
+    float a0 = bf16_lo(wa), a1 = bf16_hi(wa), b0 = bf16_lo(wb), b1 = bf16_hi(wb);
+    const uint16_t* nw = (hd < p.nq) ? p.q_norm : p.k_norm;
+    if (nw) {
+      const float ss = warp_sum(a0 * a0 + a1 * a1 + b0 * b0 + b1 * b1);
+      const float inv = 1.0f / sqrtf(ss * (1.0f / kHeadDim) + p.eps);
+      const uint32_t na = *reinterpret_cast<const uint32_t*>(nw + 2 * lane);
+      const uint32_t nb = *reinterpret_cast<const uint32_t*>(nw + 64 + 2 * lane);
+      a0 = bf16_to_f32(f32_to_bf16(a0 * inv * bf16_lo(na)));
+      a1 = bf16_to_f32(f32_to_bf16(a1 * inv * bf16_hi(na)));
+      b0 = bf16_to_f32(f32_to_bf16(b0 * inv * bf16_lo(nb)));
+      b1 = bf16_to_f32(f32_to_bf16(b1 * inv * bf16_hi(nb)));
+    }
+    const float4 cs = *reinterpret_cast<const float4*>(p.rope + ((size_t)pos * 64 + 2 * lane) * 2);  // c0 s0 c1 s1
+    oa = pack_bf16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
+    ob = pack_bf16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
+  }
+  uint16_t* dst;
+  if (hd < p.nq) {
+    dst = p.q_out + ((size_t)r * p.nq + hd) * kHeadDim;
+  } else {
+    const int kvh = (hd - p.nq) % p.nkv;
+    const bool is_v = hd >= p.nq + p.nkv;
+    const int blk = p.block_tables[(size_t)r * p.max_blocks + pos / kBlockSize], slot = pos % kBlockSize;
+    dst = (is_v ? p.vpool : p.kpool) + (((size_t)blk * p.nkv + kvh) * kBlockSize + slot) * kHeadDim;
+  }
+  *reinterpret_cast<uint32_t*>(dst + 2 * lane) = oa;
+  *reinterpret_cast<uint32_t*>(dst + 64 + 2 * lane) = ob;
+}
+
+int g_attn_sm_count = 0;
+
+}  // namespace
+
+cudaError_t attention_init() {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  int sms = 0;
+  e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(paged_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kAttnWarps * kAttnStages * kAttnStage);
+  if (e != cudaSuccess) return e;
+  g_attn_sm_count = sms;
+  return cudaSuccess;
+}
+
+int attention_max_work(int max_batch, int max_positions) {
+  // smallest automatic chunk is 4 tiles (64 tokens)
+  return max_batch * ((max_positions + 63) / 64 + 1);
+}
+
+AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, int sm_count, int4* work,
+                        int32_t* slot_base, int32_t* nchunks, int max_work) {
+  AttnPlan plan;
+  long long total_tiles = 0;
+  for (int r = 0; r < n; ++r) total_tiles += (lens[r] + 1 + 15) / 16;
+  int chunk_tiles;
+  if (chunk_tokens > 0) {
+    chunk_tiles = (chunk_tokens + 15) / 16;
+  } else {
+    // Largest chunk (up to 1024 tokens) that still yields about four CTAs per SM.
+    chunk_tiles = 64;
+    while (chunk_tiles > 4 && (total_tiles / chunk_tiles + n) * nkv < 4LL * sm_count) chunk_tiles >>= 1;
+  }
+  if (chunk_tiles < 1) chunk_tiles = 1;
+  int w = 0;
+  for (int r = 0; r < n; ++r) {
+    const int tiles = (lens[r] + 1 + 15) / 16;
+    slot_base[r] = w;
+    int c = 0;
+    for (int t0 = 0; t0 < tiles && w < max_work; t0 += chunk_tiles, ++c, ++w)
+      work[w] = make_int4(r, t0, t0 + chunk_tiles < tiles ? t0 + chunk_tiles : tiles, w);
+    nchunks[r] = c;
+  }
+  plan.n_work = w;
+  plan.n_slots = w;
+  plan.chunk_tiles = chunk_tiles;
+  return plan;
+}
+
+cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s) {
+  if (g_attn_sm_count == 0) {
+    cudaError_t e = attention_init();
+    if (e != cudaSuccess) return e;
+  }
+  if (a.n_work <= 0) return cudaSuccess;
+  const int G = a.nq / a.nkv;
+  if (G < 1 || G > 16 || a.nq % a.nkv) return cudaErrorInvalidValue;
+  const dim3 grid(a.n_work, a.nkv), block(kAttnThreads);
+  paged_attention_kernel<<<grid, block, kAttnWarps * kAttnStages * kAttnStage, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s) {
+  if (a.n <= 0) return cudaSuccess;
+  attention_merge_kernel<<<dim3(a.n, a.nq), kHeadDim, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_rope_append(const RopeArgs& a, cudaStream_t s) {
+  if (a.n <= 0) return cudaSuccess;
+  const int heads = a.nq + 2 * a.nkv;
+  rope_append_kernel<<<dim3((heads + 3) / 4, a.n), 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
+}  // namespace q4d

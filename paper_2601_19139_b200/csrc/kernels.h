@@ -1,0 +1,96 @@
+// Host-side launch interface of the q4decode kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace q4d {
+
+constexpr int kMaxBatch = 16;
+constexpr int kHeadDim = 128;
+constexpr int kBlockSize = 16;
+
+// ---- 4-bit skinny GEMM ------------------------------------------------------------
+enum GemmPrologue { PRO_PLAIN = 0, PRO_SILU_MUL = 1 };
+enum GemmEpilogue { EPI_BF16 = 0, EPI_RESIDUAL = 1, EPI_F32 = 2 };
+
+struct GemmArgs {
+  const uint32_t* qw;      // [N][K/8]
+  const uint16_t* scales;  // [N][K/64]
+  const uint16_t* biases;  // [N][K/64]
+  int N, K;
+  const uint16_t* x;  // bf16 [n][x_stride]
+  int x_stride;
+  int n;
+  int prologue, epilogue;
+  void* out;
+  int out_stride;
+  float* partial;  // split-K partial sums
+  size_t partial_bytes;
+  int* counters;  // zero between launches
+  int counters_len;
+};
+
+// Bytes of split-K scratch a GEMM of this shape may use (upper bound over batch sizes).
+size_t gemm_partial_bytes(int N, int K);
+int gemm_counters_needed(int N);
+cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s);
+cudaError_t gemm_init();  // sets the dynamic shared memory limits once per process/device
+
+// ---- paged decode attention -------------------------------------------------------
+struct AttnPlan {   // filled on the host from the request lengths
+  int n_work;       // (request, chunk) items
+  int n_slots;      // partial-result slots = n_work
+  int chunk_tiles;  // tiles (16 tokens) per chunk
+};
+// work: int4 {request, first tile, end tile, slot}; slot_base/nchunks per request.
+AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, int sm_count, int4* work,
+                        int32_t* slot_base, int32_t* nchunks, int max_work);
+int attention_max_work(int max_batch, int max_positions);
+
+struct AttnArgs {
+  const uint16_t* q;  // [n][nq][128]
+  const uint16_t* kpool;
+  const uint16_t* vpool;  // this layer: [blocks][nkv][16][128]
+  const int32_t* block_tables;
+  const int32_t* lens;
+  const int4* work;
+  const int32_t* slot_base;
+  const int32_t* nchunks;
+  int n_work, n, nq, nkv, max_blocks;
+  float* part_acc;  // [slots][nq][128]
+  float* part_ml;   // [slots][nq][2]
+  uint16_t* out;    // [n][nq][128]
+};
+cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s);
+cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s);
+cudaError_t attention_init();
+
+struct RopeArgs {
+  const uint16_t* qkv;
+  const uint16_t* q_norm;
+  const uint16_t* k_norm;
+  float eps;
+  const float* rope;
+  int n, nq, nkv;
+  const int32_t* lens;
+  const int32_t* block_tables;
+  int max_blocks;
+  uint16_t* kpool;
+  uint16_t* vpool;
+  uint16_t* q_out;
+};
+cudaError_t launch_rope_append(const RopeArgs& a, cudaStream_t s);
+
+// ---- small kernels ----------------------------------------------------------------
+cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,
+                         const int32_t* tokens, int n, uint16_t* x, cudaStream_t s);
+cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int n, int H, uint16_t* y,
+                           cudaStream_t s);
+cudaError_t launch_argmax(const float* logits, int n, int vocab, int32_t* next, cudaStream_t s);
+cudaError_t launch_dequant(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int N, int K,
+                           float* out, cudaStream_t s);
+cudaError_t launch_kv_gather(const uint16_t* kpool, const uint16_t* vpool, int nkv, const int32_t* block_table,
+                             int len, uint16_t* k_out, uint16_t* v_out, cudaStream_t s);
+
+}  // namespace q4d
