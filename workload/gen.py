@@ -200,19 +200,33 @@ class ChurnScript:
         self.next_rid = 0
         self.step = 0
         self.active = []
+        self.pending = []  # the queue Q of Algorithm 1: requests whose prefilled KV is already in the pool
         self.events = []  # ("admit", rid, len) / ("release", rid) since the last step
         for length in draw_lengths(n, lo, hi, self.rng, log_uniform):
             self._admit(int(length))
 
-    def _admit(self, length):
+    def _make_request(self, length):
         rid = self.next_rid
         self.next_rid += 1
         nblk = (length + 1 + self.bs - 1) // self.bs
         blocks = self.alloc.alloc(nblk)
         fill_blocks(self.pool, blocks, self.seed, "kv", rid)
         tok = int(self.rng.integers(0, self.shape.vocab))
-        self.active.append(Request(rid, length, blocks, tok))
-        self.events.append(("admit", rid, length))
+        return Request(rid, length, blocks, tok)
+
+    def _admit(self, length):
+        r = self.pending.pop(0) if self.pending else self._make_request(length)
+        self.active.append(r)
+        self.events.append(("admit", r.rid, r.length))
+
+    def prepare_pending(self, steps):
+        """Create ahead of time the requests that will be admitted during the next `steps` steps, so that
+        admitting them later is bookkeeping only (their prefilled KV is written now)."""
+        if not self.churn_every:
+            return
+        due = sum(1 for s in range(self.step + 1, self.step + steps + 1) if s % self.churn_every == 0)
+        while len(self.pending) < due * self.churn_count:
+            self.pending.append(self._make_request(self.admit_len))
 
     def churn(self):
         """Apply the between-steps membership change due before the coming step, if any."""
