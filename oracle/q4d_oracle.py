@@ -204,6 +204,11 @@ def attention_paged(q_bits, pool, nq, nkv, bs, d, layer, lens, block_tables):
     return out
 
 
+def probe_fp32_accumulate(on):
+    """Sensitivity probe (not the definition): projections accumulate in fp32 while set."""
+    lib().orc_probe_fp32_accumulate(C.c_int(int(bool(on))))
+
+
 def num_threads():
     return int(lib().orc_num_threads())
 

@@ -162,6 +162,15 @@ def _tables(lens, nblocks, seed):
     return bt
 
 
+def _close_after_two_roundings(got_bits, want_bits, what):
+    """The head is rounded to bf16 after the norm and again after the rotation.  A one-step difference after the
+    first rounding moves the rotated value by up to one step of the larger input, which can be several steps of a
+    small output, so the bound is absolute: one bf16 step of the head's largest element; and few elements differ."""
+    got, want = orc.bf16_to_f64(got_bits), orc.bf16_to_f64(want_bits)
+    assert np.abs(got - want).max() <= 2.0 ** -7 * np.abs(want).max(), what
+    assert (got_bits != want_bits).mean() <= 0.05, what
+
+
 @pytest.mark.parametrize("nq,nkv,qk_norm", [(16, 8, True), (24, 8, False), (32, 4, True)])
 def test_rope_append_matches_oracle(q4d, nq, nkv, qk_norm):
     lens = [0, 15, 16, 100, 257]
@@ -188,10 +197,10 @@ def test_rope_append_matches_oracle(q4d, nq, nkv, qk_norm):
                 head = orc.rmsnorm(head[None], bits(qn if hd < nq else kn), 1e-6)[0]
             want = orc.rope(head, tab[l])
             if hd < nq:
-                assert_bf16_close(bits(q_out)[r, hd], want, max_mismatch_frac=0.05, what="q")
+                _close_after_two_roundings(bits(q_out)[r, hd], want, "q")
             else:
                 blk, slot = bt[r, l // 16], l % 16
-                assert_bf16_close(after[0, blk, hd - nq, slot], want, max_mismatch_frac=0.05, what="k")
+                _close_after_two_roundings(after[0, blk, hd - nq, slot], want, "k")
                 touched[0, blk, hd - nq, slot] = True
         for hv in range(nkv):
             blk, slot = bt[r, l // 16], l % 16
