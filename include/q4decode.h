@@ -224,6 +224,27 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
                 int32_t n, int32_t prologue, int32_t epilogue, void* out, int32_t out_stride,
                 void* scratch, void* cuda_stream);
 
+/* The same projection for callers that may not allocate device memory at all (the paper has no
+ * counterpart; this is a deployment convenience).  Typical users: a plugin running inside a host
+ * process that has given all device memory to its own arena, code called from an allocator or
+ * memory-pool callback, or a serving loop where cudaMalloc is banned because it synchronises the
+ * device.  Arguments and results are those of q4d_q4_gemm without `scratch`: the split-K scratch is
+ * a fixed array inside the library (q4d_noalloc_max_scratch_bytes() = 8 MiB of partial sums plus
+ * 4096 row-block counters) that every GPU holds from the moment the library is loaded until the
+ * process exits.  The call allocates and frees nothing.
+ *  - Projections whose split-K partial sums exceed the array are refused with
+ *    WORKSPACE_TOO_SMALL (for example a 151936 x 4096 LM head at batch 16); use q4d_q4_gemm then.
+ *  - The first call on each device looks up the array's device address; make that first call
+ *    outside any stream capture, with the device current.
+ *  - Every call reuses the same array and finds in it what the previous call left; the counters are
+ *    cleared on the stream before each launch.  Calls whose kernels can overlap on the GPU (different
+ *    streams without an ordering between them) race on the array: keep them on one stream or order
+ *    them with events. */
+int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, int32_t x_stride,
+                        int32_t n, int32_t prologue, int32_t epilogue, void* out, int32_t out_stride,
+                        void* cuda_stream);
+size_t q4d_noalloc_max_scratch_bytes(void);
+
 /* y = bf16(x * rsqrt(mean(x^2) + eps) * w), rows of length H. */
 int q4d_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int32_t n, int32_t H, uint16_t* y,
                 void* cuda_stream);

@@ -22,6 +22,7 @@ EXPORTS = [
     "q4d_kv_pool_create", "q4d_kv_pool_destroy", "q4d_request_admit", "q4d_request_release", "q4d_request_len",
     "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_profile_enable",
     "q4d_profile_read", "q4d_launch_count", "q4d_step_io_bytes", "q4d_op_scratch_bytes", "q4d_q4_gemm",
+    "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
     "q4d_rmsnorm", "q4d_embed", "q4d_rope_append", "q4d_paged_attention", "q4d_argmax", "q4d_debug_dequant",
     "q4d_debug_kv_gather",
 ]
@@ -71,6 +72,7 @@ def lib():
         L.q4d_kv_pool_bytes.restype = C.c_size_t
         L.q4d_op_scratch_bytes.restype = C.c_size_t
         L.q4d_launch_count.restype = C.c_int64
+        L.q4d_noalloc_max_scratch_bytes.restype = C.c_size_t
         _LIB = L
     return _LIB
 
@@ -257,6 +259,17 @@ def q4_gemm(w, x, n, prologue=0, epilogue=0, out=None, stream=None):
     _check(lib().q4d_q4_gemm(C.byref(qt), C.c_int32(N), C.c_int32(K), _ptr(x), C.c_int32(x.stride(0)), C.c_int32(n),
                              C.c_int32(prologue), C.c_int32(epilogue), _ptr(out), C.c_int32(out.stride(0)),
                              _ptr(op_scratch(x.device)), _stream(stream)))
+    return out
+
+
+def q4_gemm_noalloc(w, x, n, out, prologue=0, epilogue=0, stream=None):
+    """q4d_q4_gemm_noalloc: like q4_gemm but with the library's built-in scratch; `out` must be preallocated."""
+    q = w[0]
+    N, K = q.shape[0], q.shape[1] * 8
+    qt = _qt(w)
+    _check(lib().q4d_q4_gemm_noalloc(C.byref(qt), C.c_int32(N), C.c_int32(K), _ptr(x), C.c_int32(x.stride(0)),
+                                     C.c_int32(n), C.c_int32(prologue), C.c_int32(epilogue), _ptr(out),
+                                     C.c_int32(out.stride(0)), _stream(stream)))
     return out
 
 

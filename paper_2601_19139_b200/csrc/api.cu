@@ -347,6 +347,9 @@ extern "C" {
 
 const char* q4d_last_error(void) { return g_last_error.c_str(); }
 
+// Lets the other translation units of the library record an error message.
+int q4d_internal_fail(int code, const char* msg) { return fail(code, "%s", msg); }
+
 size_t q4d_model_workspace_bytes(const q4d_shape* shape) {
   std::string why;
   if (!shape || !shape_supported(*shape, &why)) {

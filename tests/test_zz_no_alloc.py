@@ -1,0 +1,67 @@
+"""The no-allocation GEMM entry point, q4d_q4_gemm_noalloc.
+
+It exists for callers that cannot allocate device memory when they need a projection (a plugin whose
+host owns all device memory, code inside an allocator callback, a loop where cudaMalloc's device-wide
+synchronisation is not acceptable).  Its scratch is an array built into the library, shared by all calls,
+so the test calls it twice in a row with different shapes and checks each result against the ordinary
+entry point q4d_q4_gemm, which runs the same kernel on caller-provided scratch: the results must be
+identical.  This file sorts last so that a run stopping at the first failure has run everything else.
+"""
+import numpy as np
+import pytest
+import torch
+
+from workload import gen
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q4d():
+    from paper_2601_19139_b200 import binding, build
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _x(n, K, seed):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return torch.randn(n, K, generator=g, device="cuda").to(torch.bfloat16)
+
+
+def test_noalloc_gemm_equals_the_scratch_taking_entry_point_twice_in_a_row(q4d):
+    # outputs are allocated before the calls under test: the entry point itself must allocate nothing
+    cases = [(4096, 4096, 16, 2), (1024, 3072, 5, 0)]     # split-K in both; f32 then bf16 epilogue
+    prepared = []
+    for i, (N, K, n, epi) in enumerate(cases):
+        w = gen.random_q4(N, K, "cuda", "noalloc", i)
+        x = _x(n, K, 40 + i)
+        out = torch.full((n, N), float("nan"), dtype=torch.float32 if epi == 2 else torch.bfloat16, device="cuda")
+        prepared.append((w, x, n, epi, out))
+    torch.cuda.synchronize()
+    before = torch.cuda.memory_allocated()
+    for w, x, n, epi, out in prepared:                     # two calls in a row on the shared array
+        q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before
+    for w, x, n, epi, out in prepared:
+        want = q4d.q4_gemm(w, x, n, epilogue=epi)
+        torch.cuda.synchronize()
+        assert torch.equal(out, want)
+    # and again in the other order: what the previous call left in the array must not matter
+    for w, x, n, epi, out in reversed(prepared):
+        out.fill_(float("nan"))
+        q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
+        torch.cuda.synchronize()
+        assert torch.equal(out, q4d.q4_gemm(w, x, n, epilogue=epi))
+
+
+def test_noalloc_gemm_refuses_shapes_beyond_its_array(q4d):
+    N, K, n = 151936, 4096, 16
+    w = gen.random_q4(N, K, "cuda", "noalloc-big")
+    x = _x(n, K, 50)
+    out = torch.zeros(n, N, dtype=torch.float32, device="cuda")
+    with pytest.raises(q4d.Q4dError) as ei:
+        q4d.q4_gemm_noalloc(w, x, n, out, epilogue=2)
+    assert ei.value.code == -8 and "scratch" in str(ei.value)
+    assert q4d.lib().q4d_noalloc_max_scratch_bytes() == 8 << 20
