@@ -229,10 +229,11 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
  * process that has given all device memory to its own arena, code called from an allocator or
  * memory-pool callback, or a serving loop where cudaMalloc is banned because it synchronises the
  * device.  Arguments and results are those of q4d_q4_gemm without `scratch`: the split-K scratch is
- * a fixed array inside the library (q4d_noalloc_max_scratch_bytes() = 8 MiB of partial sums plus
- * 4096 row-block counters) that every GPU holds from the moment the library is loaded until the
- * process exits.  The call allocates and frees nothing.
- *  - Projections whose split-K partial sums exceed the array are refused with
+ * a fixed array inside the library (q4d_noalloc_max_scratch_bytes() = 8 MiB of partial sums, plus
+ * 4096 row-block counters and 0.6 MiB in which the activations are rearranged for the kernel) that
+ * every GPU holds from the moment the library is loaded until the process exits.  The call allocates
+ * and frees nothing.
+ *  - Projections whose split-K partial sums exceed the array, or with K > 16384, are refused with
  *    WORKSPACE_TOO_SMALL (for example a 151936 x 4096 LM head at batch 16); use q4d_q4_gemm then.
  *  - The first call on each device looks up the array's device address; make that first call
  *    outside any stream capture, with the device current.
@@ -276,6 +277,14 @@ int q4d_paged_attention(const uint16_t* q, const uint16_t* pool_layer_k, const u
 int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, void* cuda_stream);
 
 /* ---- parity exports ----------------------------------------------------- */
+
+/* Layers [layer_begin, layer_end) of the step, exactly as q4d_decode_step launches them (including the append of
+ * K, V at each request's current length), starting from the hidden state x_in bf16 [n][hidden] (device) and
+ * returning the hidden state after the last of them in x_out.  Request lengths do not change.  Used to compare
+ * single layers of the production path with the oracle from identical inputs. */
+int q4d_debug_run_layers(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
+                         const int32_t* block_tables, int32_t max_blocks, int32_t layer_begin, int32_t layer_end,
+                         const uint16_t* x_in_device, uint16_t* x_out_device, void* cuda_stream);
 
 /* out f32 [N][K] = the dequantised weights (bit-exact definition above). */
 int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out_device, void* cuda_stream);

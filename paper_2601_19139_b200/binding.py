@@ -24,7 +24,7 @@ EXPORTS = [
     "q4d_profile_read", "q4d_launch_count", "q4d_step_io_bytes", "q4d_op_scratch_bytes", "q4d_q4_gemm",
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
     "q4d_rmsnorm", "q4d_embed", "q4d_rope_append", "q4d_paged_attention", "q4d_argmax", "q4d_debug_dequant",
-    "q4d_debug_kv_gather",
+    "q4d_debug_kv_gather", "q4d_debug_run_layers",
 ]
 
 
@@ -336,3 +336,13 @@ def debug_kv_gather(pool, layer, block_table_device, length, stream=None):
     _check(lib().q4d_debug_kv_gather(pool.handle, C.c_int32(layer), _ptr(block_table_device), C.c_int32(length),
                                      _ptr(k), _ptr(v), _stream(stream)))
     return k, v
+
+
+def debug_run_layers(model, pool, request_ids, block_tables, layer_begin, layer_end, x_in, stream=None):
+    """q4d_debug_run_layers: layers [layer_begin, layer_end) of the production path from the hidden state x_in."""
+    ids, bt = _step_args(request_ids, block_tables)
+    x_out = torch.empty_like(x_in)
+    _check(lib().q4d_debug_run_layers(model.handle, pool.handle, C.c_int32(ids.size), _ptr(ids), _ptr(bt),
+                                      C.c_int32(bt.shape[1]), C.c_int32(layer_begin), C.c_int32(layer_end),
+                                      _ptr(x_in), _ptr(x_out), _stream(stream)))
+    return x_out

@@ -2,6 +2,7 @@
 // stream-ordered launch sequence of one decode step.
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -34,6 +35,8 @@ int fail_cuda(cudaError_t e, const char* what) {
   return fail(Q4D_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+bool g_pdl = true;
+
 constexpr size_t kAlign = 256;
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
@@ -56,9 +59,11 @@ struct MetaLayout {
 };
 
 struct Workspace {
-  size_t x, y, qkv, qbuf, attn, gu, logits, next, gemm_partial, gemm_partial_bytes, counters, part_acc, part_ml,
-      meta, bytes;
-  int counters_len;
+  // x: residual stream (plain).  yp/ys, ap/as, hp/hs: GEMM operands in fragment order with their group sums
+  // (normed hidden state, attention output, silu(gate)*up).
+  size_t x, yp, ys, qkv, qbuf, ap, as, hp, hs, logits, next, amax, gemm_partial, gemm_partial_bytes, counters,
+      part_acc, part_ml, meta, bytes;
+  int counters_len, amax_blocks;
 };
 
 bool shape_supported(const q4d_shape& s, std::string* why) {
@@ -92,25 +97,31 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   };
   const size_t B = kMaxBatch;
   const int nqkv = (s.n_q_heads + 2 * s.n_kv_heads) * kHeadDim;
+  const size_t qdim = (size_t)s.n_q_heads * kHeadDim;
   w.x = take(B * s.hidden * 2);
-  w.y = take(B * s.hidden * 2);
+  w.yp = take(B * s.hidden * 2);
+  w.ys = take((size_t)(s.hidden / 64) * 16 * 4);
   w.qkv = take(B * nqkv * 2);
-  w.qbuf = take(B * s.n_q_heads * kHeadDim * 2);
-  w.attn = take(B * s.n_q_heads * kHeadDim * 2);
-  w.gu = take(B * 2 * (size_t)s.mlp_inter * 2);
+  w.qbuf = take(B * qdim * 2);
+  w.ap = take(B * qdim * 2);
+  w.as = take((qdim / 64) * 16 * 4);
+  w.hp = take(B * (size_t)s.mlp_inter * 2);
+  w.hs = take((size_t)(s.mlp_inter / 64) * 16 * 4);
   w.logits = take(B * (size_t)s.vocab * 4);
   w.next = take(B * 4);
+  w.amax_blocks = (s.vocab + 127) / 128 + 1;
+  w.amax = take((size_t)w.amax_blocks * 16 * sizeof(float2));
   size_t pb = 0;
   int cl = 0;
-  auto gemm = [&](int N, int K) {
-    pb = std::max(pb, gemm_partial_bytes(N, K));
+  auto gemm = [&](int N, int K, int epi) {
+    pb = std::max(pb, gemm_partial_bytes(N, K, epi));
     cl = std::max(cl, gemm_counters_needed(N));
   };
-  gemm(nqkv, s.hidden);
-  gemm(s.hidden, s.n_q_heads * kHeadDim);
-  gemm(2 * s.mlp_inter, s.hidden);
-  gemm(s.hidden, s.mlp_inter);
-  gemm(s.vocab, s.hidden);
+  gemm(nqkv, s.hidden, EPI_BF16);
+  gemm(s.hidden, s.n_q_heads * kHeadDim, EPI_RESIDUAL);
+  gemm(2 * s.mlp_inter, s.hidden, EPI_SILU_PACK);
+  gemm(s.hidden, s.mlp_inter, EPI_RESIDUAL);
+  gemm(s.vocab, s.hidden, EPI_F32);
   w.gemm_partial_bytes = pb;
   w.gemm_partial = take(pb);
   w.counters_len = cl;
@@ -192,12 +203,13 @@ cudaError_t timed(q4d_model* m, int cls, cudaStream_t s, F&& f) {
   return e;
 }
 
-GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint16_t* x, int x_stride, int n, int pro,
+GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint16_t* xp, const float* xs, int n,
                    int epi, void* out, int out_stride) {
   GemmArgs a;
   a.qw = t.q, a.scales = t.scales, a.biases = t.biases;
-  a.N = N, a.K = K, a.x = x, a.x_stride = x_stride, a.n = n, a.prologue = pro, a.epilogue = epi;
+  a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n, a.epilogue = epi;
   a.out = out, a.out_stride = out_stride;
+  a.out_xp = nullptr, a.out_xs = nullptr, a.argmax_partial = nullptr;
   a.partial = at<float>(m, m->lay.gemm_partial), a.partial_bytes = m->lay.gemm_partial_bytes;
   a.counters = at<int>(m, m->lay.counters), a.counters_len = m->lay.counters_len;
   return a;
@@ -205,15 +217,24 @@ GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint1
 
 bool qt_ok(const q4d_qtensor& t) { return t.q && t.scales && t.biases; }
 
+// The launch sequence of a step.  A whole step embeds the tokens, runs every layer and the head, and advances the
+// requests.  The parity export runs only layers [layer_begin, layer_end) from a given hidden state (x_in) and
+// returns the hidden state (x_out) without advancing anything.
+struct LayerRange {
+  int begin, end;
+  const uint16_t* x_in;
+  uint16_t* x_out;
+};
+
 int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* tokens_host,
               const int32_t* tokens_dev, const int32_t* bt, int32_t max_blocks, int32_t* next_dev, float* logits_dev,
-              cudaStream_t s) {
+              cudaStream_t s, const LayerRange* range = nullptr) {
   if (!m || !pool || pool->model != m) return fail(Q4D_ERR_INVALID_ARG, "decode_step: model/pool mismatch or NULL");
   if (n < 0) return fail(Q4D_ERR_INVALID_ARG, "decode_step: n < 0");
   if (n == 0) return Q4D_OK;
   if (n > m->sh.max_batch)
     return fail(Q4D_ERR_BATCH_TOO_LARGE, "decode_step: n = %d exceeds max_batch %d", n, m->sh.max_batch);
-  if (!ids || (!tokens_host && !tokens_dev) || !bt || !next_dev || max_blocks < 1)
+  if (!ids || !bt || max_blocks < 1 || (!range && ((!tokens_host && !tokens_dev) || !next_dev)))
     return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL argument");
   const q4d_shape& sh = m->sh;
 
@@ -287,13 +308,18 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   const int H = sh.hidden, nq = sh.n_q_heads, nkv = sh.n_kv_heads, I = sh.mlp_inter, V = sh.vocab;
   const int nqkv = (nq + 2 * nkv) * kHeadDim;
   uint16_t* x = at<uint16_t>(m, m->lay.x);
-  uint16_t* y = at<uint16_t>(m, m->lay.y);
+  uint16_t* yp = at<uint16_t>(m, m->lay.yp);
+  float* ys = at<float>(m, m->lay.ys);
   uint16_t* qkv = at<uint16_t>(m, m->lay.qkv);
   uint16_t* qbuf = at<uint16_t>(m, m->lay.qbuf);
-  uint16_t* attn = at<uint16_t>(m, m->lay.attn);
-  uint16_t* gu = at<uint16_t>(m, m->lay.gu);
+  uint16_t* ap = at<uint16_t>(m, m->lay.ap);
+  float* as = at<float>(m, m->lay.as);
+  uint16_t* hp = at<uint16_t>(m, m->lay.hp);
+  float* hs = at<float>(m, m->lay.hs);
+  float2* amax = at<float2>(m, m->lay.amax);
   float* logits = logits_dev ? logits_dev : at<float>(m, m->lay.logits);
   const size_t layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
+  const int qdim = nq * kHeadDim;
 
 #define Q4D_LAUNCH(cls, expr)                                                 \
   do {                                                                        \
@@ -301,14 +327,18 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     if (le != cudaSuccess) return fail_cuda(le, #cls);                        \
   } while (0)
 
-  Q4D_LAUNCH(Q4D_K_EMBED, launch_embed(m->w.embed.q, m->w.embed.scales, m->w.embed.biases, V, H, d_tokens, n, x, s));
-  for (int l = 0; l < sh.n_layers; ++l) {
+  if (range) {
+    cudaError_t ce = cudaMemcpyAsync(x, range->x_in, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
+    if (ce != cudaSuccess) return fail_cuda(ce, "hidden state copy");
+  } else {
+    Q4D_LAUNCH(Q4D_K_EMBED, launch_embed(m->w.embed.q, m->w.embed.scales, m->w.embed.biases, V, H, d_tokens, n, x, s));
+  }
+  for (int l = range ? range->begin : 0; l < (range ? range->end : sh.n_layers); ++l) {
     const q4d_layer_weights& lw = m->layers[l];
     uint16_t* kpool = pool->mem + (size_t)(2 * l) * layer_elems;
     uint16_t* vpool = kpool + layer_elems;
-    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, y, s));
-    Q4D_LAUNCH(Q4D_K_GEMM_QKV,
-               launch_q4_gemm(gemm_args(m, lw.wqkv, nqkv, H, y, H, n, PRO_PLAIN, EPI_BF16, qkv, nqkv), s));
+    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+    Q4D_LAUNCH(Q4D_K_GEMM_QKV, launch_q4_gemm(gemm_args(m, lw.wqkv, nqkv, H, yp, ys, n, EPI_BF16, qkv, nqkv), s));
     RopeArgs ra;
     ra.qkv = qkv, ra.q_norm = sh.qk_norm ? lw.q_norm : nullptr, ra.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
     ra.eps = sh.rms_eps, ra.rope = m->w.rope_cos_sin, ra.n = n, ra.nq = nq, ra.nkv = nkv, ra.lens = d_lens;
@@ -320,21 +350,28 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     aa.slot_base = reinterpret_cast<const int32_t*>(dmeta + ml.off_slot_base);
     aa.nchunks = reinterpret_cast<const int32_t*>(dmeta + ml.off_nchunks);
     aa.n_work = plan.n_work, aa.n = n, aa.nq = nq, aa.nkv = nkv, aa.max_blocks = ml.max_blocks_cap;
-    aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml), aa.out = attn;
+    aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml);
+    aa.out = nullptr, aa.out_xp = ap, aa.out_xs = as;
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
     Q4D_LAUNCH(Q4D_K_ATTN_MERGE, launch_attention_merge(aa, s));
-    Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, nq * kHeadDim, attn, nq * kHeadDim, n, PRO_PLAIN,
-                                                      EPI_RESIDUAL, x, H), s));
-    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, y, s));
-    Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP,
-               launch_q4_gemm(gemm_args(m, lw.w_gate_up, 2 * I, H, y, H, n, PRO_PLAIN, EPI_BF16, gu, 2 * I), s));
-    Q4D_LAUNCH(Q4D_K_GEMM_DOWN,
-               launch_q4_gemm(gemm_args(m, lw.w_down, H, I, gu, 2 * I, n, PRO_SILU_MUL, EPI_RESIDUAL, x, H), s));
+    Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
+    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+    GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
+    gu.out_xp = hp, gu.out_xs = hs;
+    Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
+    Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
   }
-  Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, y, s));
-  Q4D_LAUNCH(Q4D_K_LM_HEAD,
-             launch_q4_gemm(gemm_args(m, m->w.lm_head, V, H, y, H, n, PRO_PLAIN, EPI_F32, logits, V), s));
-  Q4D_LAUNCH(Q4D_K_ARGMAX, launch_argmax(logits, n, V, next_dev, s));
+  if (range) {
+    cudaError_t ce = cudaMemcpyAsync(range->x_out, x, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
+    return ce == cudaSuccess ? Q4D_OK : fail_cuda(ce, "hidden state copy");
+  }
+  Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+  GemmArgs lm = gemm_args(m, m->w.lm_head, V, H, yp, ys, n, EPI_F32, logits, V);
+  lm.argmax_partial = amax;
+  const int lm_blocks = gemm_row_blocks(V, H, n, EPI_F32);
+  if (lm_blocks > m->lay.amax_blocks) return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "decode_step: argmax scratch too small");
+  Q4D_LAUNCH(Q4D_K_LM_HEAD, launch_q4_gemm(lm, s));
+  Q4D_LAUNCH(Q4D_K_ARGMAX, launch_argmax_finish(amax, lm_blocks, n, next_dev, s));
 #undef Q4D_LAUNCH
 
   for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
@@ -342,6 +379,11 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
 }
 
 }  // namespace
+
+namespace q4d {
+void set_pdl_enabled(bool on) { g_pdl = on; }
+bool pdl_enabled() { return g_pdl; }
+}  // namespace q4d
 
 extern "C" {
 
@@ -379,6 +421,7 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   }
   MetaLayout ml;
   ml.init(shape->max_positions);
+  if (const char* v = getenv("Q4D_NO_PDL")) set_pdl_enabled(v[0] == '0');
   cudaError_t e = gemm_init();
   if (e == cudaSuccess) e = attention_init();
   if (e != cudaSuccess) return fail_cuda(e, "kernel init");
@@ -566,9 +609,13 @@ constexpr size_t kOpGemmPartial = 48ull << 20;
 constexpr size_t kOpAttnMeta = 1ull << 20;
 constexpr size_t kOpPartAcc = 64ull << 20;
 constexpr size_t kOpPartMl = 1ull << 20;
+constexpr int kOpMaxK = 32768;                         // widest operand the pack buffers hold
+constexpr size_t kOpPackXp = (size_t)16 * kOpMaxK * 2;  // fragment-ordered operand
+constexpr size_t kOpPackXs = (size_t)(kOpMaxK / 64) * 16 * 4;
+constexpr size_t kOpPackOff = kOpCounters + kOpGemmPartial + kOpAttnMeta + kOpPartAcc + kOpPartMl;
 }  // namespace
 
-size_t q4d_op_scratch_bytes(void) { return kOpCounters + kOpGemmPartial + kOpAttnMeta + kOpPartAcc + kOpPartMl; }
+size_t q4d_op_scratch_bytes(void) { return kOpPackOff + kOpPackXp + kOpPackXs; }
 
 int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, int32_t x_stride, int32_t n,
                 int32_t prologue, int32_t epilogue, void* out, int32_t out_stride, void* scratch, void* stream) {
@@ -576,21 +623,29 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
   if (n < 0 || n > kMaxBatch || N < 1 || K < 256 || K % 256 || x_stride % 8 || prologue < 0 || prologue > 1 ||
       epilogue < 0 || epilogue > 2)
     return fail(Q4D_ERR_INVALID_ARG, "q4_gemm: bad shape (K must be a multiple of 256, n <= 16)");
-  if (gemm_partial_bytes(N, K) > kOpGemmPartial || (size_t)gemm_counters_needed(N) * 4 > kOpCounters)
+  if (K > kOpMaxK || gemm_partial_bytes(N, K, epilogue) > kOpGemmPartial ||
+      (size_t)gemm_counters_needed(N) * 4 > kOpCounters)
     return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "q4_gemm: shape needs more scratch than q4d_op_scratch_bytes provides");
-  GemmArgs a;
-  a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.x = x, a.x_stride = x_stride, a.n = n;
-  a.prologue = prologue, a.epilogue = epilogue, a.out = out, a.out_stride = out_stride;
   unsigned char* sc = static_cast<unsigned char*>(scratch);
+  uint16_t* xp = reinterpret_cast<uint16_t*>(sc + kOpPackOff);
+  float* xs = reinterpret_cast<float*>(sc + kOpPackOff + kOpPackXp);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, st);
+  if (e != cudaSuccess) return fail_cuda(e, "q4_gemm (operand)");
+  GemmArgs a;
+  a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;
+  a.epilogue = epilogue, a.out = out, a.out_stride = out_stride;
+  a.out_xp = nullptr, a.out_xs = nullptr, a.argmax_partial = nullptr;
   a.counters = reinterpret_cast<int*>(sc), a.counters_len = (int)(kOpCounters / 4);
   a.partial = reinterpret_cast<float*>(sc + kOpCounters), a.partial_bytes = kOpGemmPartial;
-  cudaError_t e = launch_q4_gemm(a, static_cast<cudaStream_t>(stream));
+  e = launch_q4_gemm(a, st);
   return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "q4_gemm");
 }
 
 int q4d_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int32_t n, int32_t H, uint16_t* y, void* stream) {
-  if (!x || !w || !y || n < 0 || H < 2 || H % 2) return fail(Q4D_ERR_INVALID_ARG, "rmsnorm: bad argument");
-  cudaError_t e = launch_rmsnorm(x, w, eps, n, H, y, static_cast<cudaStream_t>(stream));
+  if (!x || !w || !y || n < 0 || H < 64 || H % 64 || H > 16384)
+    return fail(Q4D_ERR_INVALID_ARG, "rmsnorm: bad argument (H must be a multiple of 64, at most 16384)");
+  cudaError_t e = launch_rmsnorm(x, w, eps, n, H, y, nullptr, nullptr, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "rmsnorm");
 }
 
@@ -648,7 +703,7 @@ int q4d_paged_attention(const uint16_t* q, const uint16_t* kpool, const uint16_t
   a.n_work = plan.n_work, a.n = n, a.nq = nq, a.nkv = nkv, a.max_blocks = max_blocks;
   a.part_acc = reinterpret_cast<float*>(sc + kOpAttnMeta);
   a.part_ml = reinterpret_cast<float*>(sc + kOpAttnMeta + kOpPartAcc);
-  a.out = out;
+  a.out = out, a.out_xp = nullptr, a.out_xs = nullptr;
   e = launch_paged_attention(a, s);
   if (e == cudaSuccess) e = launch_attention_merge(a, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);  // the host work list must outlive the copy
@@ -659,6 +714,16 @@ int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, voi
   if (!logits || !next || n < 0 || vocab < 1) return fail(Q4D_ERR_INVALID_ARG, "argmax: bad argument");
   cudaError_t e = launch_argmax(logits, n, vocab, next, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "argmax");
+}
+
+int q4d_debug_run_layers(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* bt,
+                         int32_t max_blocks, int32_t layer_begin, int32_t layer_end, const uint16_t* x_in,
+                         uint16_t* x_out, void* stream) {
+  if (!m || !x_in || !x_out || layer_begin < 0 || layer_end > m->sh.n_layers || layer_begin > layer_end)
+    return fail(Q4D_ERR_INVALID_ARG, "debug_run_layers: bad argument");
+  const LayerRange range{layer_begin, layer_end, x_in, x_out};
+  return step_impl(m, pool, n, ids, nullptr, nullptr, bt, max_blocks, nullptr, nullptr,
+                   static_cast<cudaStream_t>(stream), &range);
 }
 
 int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out, void* stream) {

@@ -17,6 +17,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace q4d {
 
@@ -35,6 +36,7 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
   const int G = p.nq / p.nkv;
   const int h = blockIdx.y;
 
+  grid_launch_dependents();
   grid_dependency_wait();
 
   for (int item = blockIdx.x; item < p.n_work; item += gridDim.x) {
@@ -215,25 +217,52 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
 }
 
 // out[r][a] = bf16(sum_c 2^(m_c - M) acc_c / sum_c 2^(m_c - M) l_c) over the request's chunks, in chunk order.
-__global__ void __launch_bounds__(kHeadDim) attention_merge_kernel(const AttnArgs p) {
+// 16 threads per head, 8 consecutive elements each; a CTA of 128 threads takes 8 heads.  Writes the plain
+// layout and/or the fragment-ordered operand of the O projection (K = nq * 128) with its group sums.
+__global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs p) {
+  grid_launch_dependents();
   grid_dependency_wait();
-  const int r = blockIdx.x, a = blockIdx.y, d = threadIdx.x;
+  const int r = blockIdx.x, a = blockIdx.y * 8 + (threadIdx.x >> 4), ch = threadIdx.x & 15;
+  const bool valid = a < p.nq;
   const int s0 = p.slot_base[r], nc = p.nchunks[r];
-  float M = -INFINITY;
-  for (int c = 0; c < nc; ++c) M = fmaxf(M, p.part_ml[((size_t)(s0 + c) * p.nq + a) * 2]);
-  float num = 0.0f, den = 0.0f;
-  for (int c = 0; c < nc; ++c) {
-    const size_t qh = (size_t)(s0 + c) * p.nq + a;
-    const float e = exp2f(p.part_ml[qh * 2] - M);
-    num = fmaf(e, p.part_acc[qh * kHeadDim + d], num);
-    den = fmaf(e, p.part_ml[qh * 2 + 1], den);
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float den = 0.0f;
+  if (valid) {
+    float M = -INFINITY;
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, p.part_ml[((size_t)(s0 + c) * p.nq + a) * 2]);
+    for (int c = 0; c < nc; ++c) {
+      const size_t qh = (size_t)(s0 + c) * p.nq + a;
+      const float e = exp2f(p.part_ml[qh * 2] - M);
+      const float4 u = *reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8);
+      const float4 v = *reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8 + 4);
+      acc[0] = fmaf(e, u.x, acc[0]), acc[1] = fmaf(e, u.y, acc[1]), acc[2] = fmaf(e, u.z, acc[2]);
+      acc[3] = fmaf(e, u.w, acc[3]), acc[4] = fmaf(e, v.x, acc[4]), acc[5] = fmaf(e, v.y, acc[5]);
+      acc[6] = fmaf(e, v.z, acc[6]), acc[7] = fmaf(e, v.w, acc[7]);
+      den = fmaf(e, p.part_ml[qh * 2 + 1], den);
+    }
+  } else {
+    den = 1.0f;
   }
-  p.out[((size_t)r * p.nq + a) * kHeadDim + d] = f32_to_bf16(num / den);
+  uint4 o;
+  o.x = pack_bf16x2(acc[0] / den, acc[1] / den);
+  o.y = pack_bf16x2(acc[2] / den, acc[3] / den);
+  o.z = pack_bf16x2(acc[4] / den, acc[5] / den);
+  o.w = pack_bf16x2(acc[6] / den, acc[7] / den);
+  const float gsum = group_sum_8lanes(chunk_sum(o));  // 8 lanes = 64 elements = one group of the O projection's K
+  if (!valid) return;
+  const size_t col = (size_t)a * kHeadDim + ch * 8;
+  const size_t K = (size_t)p.nq * kHeadDim;
+  if (p.out) *reinterpret_cast<uint4*>(p.out + (size_t)r * K + col) = o;
+  if (p.out_xp) {
+    *reinterpret_cast<uint4*>(p.out_xp + (size_t)r * K + col) = permute_chunk(o);
+    if ((ch & 7) == 0) p.out_xs[(col >> 6) * 16 + r] = gsum;
+  }
 }
 
 // One warp per (request, head of qkv): optional RMSNorm over the head, rotary embedding at the
 // request's position, then q -> q_out, k and v -> the pool slot of the new token.
 __global__ void __launch_bounds__(128) rope_append_kernel(const RopeArgs p) {
+  grid_launch_dependents();
   grid_dependency_wait();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int heads = p.nq + 2 * p.nkv;
@@ -336,21 +365,18 @@ cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s) {
   const int G = a.nq / a.nkv;
   if (G < 1 || G > 16 || a.nq % a.nkv) return cudaErrorInvalidValue;
   const dim3 grid(a.n_work, a.nkv), block(kAttnThreads);
-  paged_attention_kernel<<<grid, block, kAttnWarps * kAttnStages * kAttnStage, s>>>(a);
-  return cudaGetLastError();
+  return launch_kernel(paged_attention_kernel, grid, block, kAttnWarps * kAttnStages * kAttnStage, s, a);
 }
 
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s) {
   if (a.n <= 0) return cudaSuccess;
-  attention_merge_kernel<<<dim3(a.n, a.nq), kHeadDim, 0, s>>>(a);
-  return cudaGetLastError();
+  return launch_kernel(attention_merge_kernel, dim3(a.n, (a.nq + 7) / 8), dim3(128), 0, s, a);
 }
 
 cudaError_t launch_rope_append(const RopeArgs& a, cudaStream_t s) {
   if (a.n <= 0) return cudaSuccess;
   const int heads = a.nq + 2 * a.nkv;
-  rope_append_kernel<<<dim3((heads + 3) / 4, a.n), 128, 0, s>>>(a);
-  return cudaGetLastError();
+  return launch_kernel(rope_append_kernel, dim3((heads + 3) / 4, a.n), dim3(128), 0, s, a);
 }
 
 }  // namespace q4d

@@ -63,6 +63,31 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
                : "r"(smem_u32(smem_row)));
 }
 
+// ---- fragment-ordered GEMM operand ---------------------------------------------------
+// The GEMM reads its activations as bf16 [16][K] with every aligned chunk of 8 elements stored in the order
+// {0,4,1,5,2,6,3,7} (so that a lane's 16 bytes are its B fragments of two k-steps), plus the fp32 sum of every
+// group of 64 elements, [K/64][16].  Producers build both with these helpers, always with the same summation
+// tree: ((e0+e1)+(e2+e3))+((e4+e5)+(e6+e7)) per chunk, then a pairwise tree over the 8 chunks of the group.
+__device__ __forceinline__ uint4 permute_chunk(const uint4 v) {
+  uint4 o;
+  o.x = __byte_perm(v.x, v.z, 0x5410);
+  o.y = __byte_perm(v.x, v.z, 0x7632);
+  o.z = __byte_perm(v.y, v.w, 0x5410);
+  o.w = __byte_perm(v.y, v.w, 0x7632);
+  return o;
+}
+__device__ __forceinline__ float chunk_sum(const uint4 v) {  // v in natural order
+  return ((bf16_lo(v.x) + bf16_hi(v.x)) + (bf16_lo(v.y) + bf16_hi(v.y))) +
+         ((bf16_lo(v.z) + bf16_hi(v.z)) + (bf16_lo(v.w) + bf16_hi(v.w)));
+}
+// Sum over the 8 lanes of an aligned lane group (each lane holds one chunk of the same 64-element group).
+__device__ __forceinline__ float group_sum_8lanes(float s) {
+  s += __shfl_xor_sync(0xffffffffu, s, 1);
+  s += __shfl_xor_sync(0xffffffffu, s, 2);
+  s += __shfl_xor_sync(0xffffffffu, s, 4);
+  return s;
+}
+
 // ---- warp reductions ----------------------------------------------------------------
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

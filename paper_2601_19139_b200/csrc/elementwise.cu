@@ -4,6 +4,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace q4d {
 
@@ -17,6 +18,7 @@ __device__ __forceinline__ float dequant(const uint32_t* qrow, const uint16_t* s
 // x[r][k] = bf16(w[tok_r][k]); token ids outside the vocabulary are clamped.
 __global__ void embed_kernel(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,
                              const int32_t* tokens, uint16_t* x) {
+  grid_launch_dependents();
   grid_dependency_wait();
   const int r = blockIdx.x;
   int tok = tokens[r];
@@ -38,26 +40,89 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return tot;
 }
 
-// y = bf16(x / sqrt(mean(x^2) + eps) * w); one CTA per request row.
+// y = bf16(x / sqrt(mean(x^2) + eps) * w); one CTA per request row.  The row is held in registers (up to 8 chunks
+// of 8 elements per thread: H <= 16384).  Writes y in plain layout and/or as the next GEMM's operand.
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* x, const uint16_t* w, float eps, int H,
-                                                       uint16_t* y) {
+                                                       uint16_t* y, uint16_t* yp, float* ys) {
   __shared__ float red[8];
+  grid_launch_dependents();
+  const int r = blockIdx.x, nch = H >> 3;
+  uint4 wv[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {  // norm weights do not depend on the preceding kernel
+    const int c = threadIdx.x + i * 256;
+    wv[i] = c < nch ? *reinterpret_cast<const uint4*>(w + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+  }
   grid_dependency_wait();
-  const uint16_t* xr = x + (size_t)blockIdx.x * H;
-  uint16_t* yr = y + (size_t)blockIdx.x * H;
+  uint4 xv[8];
   float ss = 0.0f;
-  for (int i = threadIdx.x * 2; i < H; i += blockDim.x * 2) {
-    const uint32_t v = *reinterpret_cast<const uint32_t*>(xr + i);
-    const float a = bf16_lo(v), b = bf16_hi(v);
-    ss = fmaf(a, a, ss);
-    ss = fmaf(b, b, ss);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = threadIdx.x + i * 256;
+    xv[i] = c < nch ? *reinterpret_cast<const uint4*>(x + (size_t)r * H + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t e[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float a = bf16_lo(e[j]), b = bf16_hi(e[j]);
+      ss = fmaf(a, a, ss);
+      ss = fmaf(b, b, ss);
+    }
   }
   ss = block_sum(ss, red);
   const float inv = 1.0f / sqrtf(ss / (float)H + eps);
-  for (int i = threadIdx.x * 2; i < H; i += blockDim.x * 2) {
-    const uint32_t v = *reinterpret_cast<const uint32_t*>(xr + i);
-    const uint32_t ww = *reinterpret_cast<const uint32_t*>(w + i);
-    *reinterpret_cast<uint32_t*>(yr + i) = pack_bf16x2(bf16_lo(v) * inv * bf16_lo(ww), bf16_hi(v) * inv * bf16_hi(ww));
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int c = threadIdx.x + i * 256;
+    if (i * 256 >= nch) break;  // uniform across the CTA
+    const uint32_t e[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w}, ww[4] = {wv[i].x, wv[i].y, wv[i].z, wv[i].w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      o[j] = pack_bf16x2(bf16_lo(e[j]) * inv * bf16_lo(ww[j]), bf16_hi(e[j]) * inv * bf16_hi(ww[j]));
+    const uint4 v = make_uint4(o[0], o[1], o[2], o[3]);
+    const float gsum = group_sum_8lanes(chunk_sum(v));  // lanes of an aligned group of 8 hold one 64-element group
+    if (c < nch) {
+      if (y) *reinterpret_cast<uint4*>(y + (size_t)r * H + c * 8) = v;
+      if (yp) {
+        *reinterpret_cast<uint4*>(yp + (size_t)r * H + c * 8) = permute_chunk(v);
+        if ((c & 7) == 0) ys[(size_t)(c >> 3) * 16 + r] = gsum;
+      }
+    }
+  }
+}
+
+// Plain activations -> the GEMM's fragment-ordered operand (optionally h = bf16(silu(gate) * up) first).
+// One thread per chunk of 8 elements; x is [n][x_stride] (with the SiLU prologue: gate at [0, K), up at [K, 2K)).
+__global__ void __launch_bounds__(256) pack_operand_kernel(const uint16_t* x, int x_stride, int K, int n, int prologue,
+                                                            uint16_t* xp, float* xs) {
+  grid_launch_dependents();
+  grid_dependency_wait();
+  const int cpr = K >> 3;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;  // cpr is a multiple of 32: warps never straddle rows
+  const int r = c / cpr, kc = c - r * cpr;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (r < n) {
+    const uint16_t* src = x + (size_t)r * x_stride + kc * 8;
+    v = *reinterpret_cast<const uint4*>(src);
+    if (prologue == PRO_SILU_MUL) {
+      const uint4 u = *reinterpret_cast<const uint4*>(src + K);
+      const uint32_t gw[4] = {v.x, v.y, v.z, v.w}, uw[4] = {u.x, u.y, u.z, u.w};
+      uint32_t hw[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float g0 = bf16_lo(gw[i]), g1 = bf16_hi(gw[i]);
+        hw[i] = pack_bf16x2((g0 / (1.0f + expf(-g0))) * bf16_lo(uw[i]), (g1 / (1.0f + expf(-g1))) * bf16_hi(uw[i]));
+      }
+      v = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+    }
+  }
+  const float gsum = group_sum_8lanes(chunk_sum(v));
+  if (r < n) {
+    *reinterpret_cast<uint4*>(xp + (size_t)r * K + kc * 8) = permute_chunk(v);
+    if ((kc & 7) == 0) xs[(size_t)(kc >> 3) * 16 + r] = gsum;
   }
 }
 
@@ -65,6 +130,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* x, const u
 __global__ void __launch_bounds__(1024) argmax_kernel(const float* logits, int vocab, int32_t* next) {
   __shared__ float sv[32];
   __shared__ int si[32];
+  grid_launch_dependents();
   grid_dependency_wait();
   const float* row = logits + (size_t)blockIdx.x * vocab;
   float best = -INFINITY;
@@ -124,22 +190,28 @@ __global__ void kv_gather_kernel(const uint16_t* kpool, const uint16_t* vpool, i
 cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,
                          const int32_t* tokens, int n, uint16_t* x, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
-  embed_kernel<<<n, 256, 0, s>>>(q, scales, biases, vocab, H, tokens, x);
-  return cudaGetLastError();
+  return launch_kernel(embed_kernel, dim3(n), dim3(256), 0, s, q, scales, biases, vocab, H, tokens, x);
 }
 
 cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int n, int H, uint16_t* y,
-                           cudaStream_t s) {
+                           uint16_t* yp, float* ys, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
-  if (H % 2) return cudaErrorInvalidValue;
-  rmsnorm_kernel<<<n, 256, 0, s>>>(x, w, eps, H, y);
-  return cudaGetLastError();
+  if (H % 64 || H > 16384 || (yp && !ys)) return cudaErrorInvalidValue;
+  return launch_kernel(rmsnorm_kernel, dim3(n), dim3(256), 0, s, x, w, eps, H, y, yp, ys);
+}
+
+cudaError_t launch_pack_operand(const uint16_t* x, int x_stride, int K, int n, int prologue, uint16_t* xp, float* xs,
+                                cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  if (K % 256 || x_stride % 8) return cudaErrorInvalidValue;
+  const int chunks = n * (K >> 3);
+  return launch_kernel(pack_operand_kernel, dim3((chunks + 255) / 256), dim3(256), 0, s, x, x_stride, K, n, prologue,
+                       xp, xs);
 }
 
 cudaError_t launch_argmax(const float* logits, int n, int vocab, int32_t* next, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
-  argmax_kernel<<<n, 1024, 0, s>>>(logits, vocab, next);
-  return cudaGetLastError();
+  return launch_kernel(argmax_kernel, dim3(n), dim3(1024), 0, s, logits, vocab, next);
 }
 
 cudaError_t launch_dequant(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int N, int K,

@@ -10,32 +10,51 @@ constexpr int kMaxBatch = 16;
 constexpr int kHeadDim = 128;
 constexpr int kBlockSize = 16;
 
-// ---- 4-bit skinny GEMM ------------------------------------------------------------
+// ---- launch helper -----------------------------------------------------------------
+// Launches with the programmatic-dependent-launch attribute when `pdl` is set: the kernel may start while its
+// predecessor on the stream drains; every kernel of the library waits (griddepcontrol.wait) before it touches
+// memory that another kernel writes.
+void set_pdl_enabled(bool on);
+bool pdl_enabled();
+
+// ---- fragment-ordered GEMM operand ---------------------------------------------------
+// xp bf16 [16][K] (chunks of 8 permuted), xs f32 [K/64][16] (group sums); see common.cuh.
 enum GemmPrologue { PRO_PLAIN = 0, PRO_SILU_MUL = 1 };
-enum GemmEpilogue { EPI_BF16 = 0, EPI_RESIDUAL = 1, EPI_F32 = 2 };
+cudaError_t launch_pack_operand(const uint16_t* x, int x_stride, int K, int n, int prologue, uint16_t* xp, float* xs,
+                                cudaStream_t s);
+
+// ---- 4-bit skinny GEMM ------------------------------------------------------------
+// EPI_SILU_PACK: the tensor has 2*I rows (gate rows then up rows); the output is the operand of the next GEMM,
+// h = bf16(silu(bf16(gate)) * bf16(up)), written in fragment order to out_xp [16][I] and out_xs [I/64][16].
+enum GemmEpilogue { EPI_BF16 = 0, EPI_RESIDUAL = 1, EPI_F32 = 2, EPI_SILU_PACK = 3 };
 
 struct GemmArgs {
   const uint32_t* qw;      // [N][K/8]
   const uint16_t* scales;  // [N][K/64]
   const uint16_t* biases;  // [N][K/64]
   int N, K;
-  const uint16_t* x;  // bf16 [n][x_stride]
-  int x_stride;
+  const uint16_t* xp;  // fragment-ordered operand
+  const float* xs;
   int n;
-  int prologue, epilogue;
+  int epilogue;
   void* out;
   int out_stride;
-  float* partial;  // split-K partial sums
+  uint16_t* out_xp;  // EPI_SILU_PACK only
+  float* out_xs;
+  float2* argmax_partial;  // EPI_F32 only, optional: [row blocks][16] = (max, index as float bits) per request
+  float* partial;          // split-K partial sums
   size_t partial_bytes;
   int* counters;  // zero between launches
   int counters_len;
 };
 
 // Bytes of split-K scratch a GEMM of this shape may use (upper bound over batch sizes).
-size_t gemm_partial_bytes(int N, int K);
+size_t gemm_partial_bytes(int N, int K, int epilogue);
 int gemm_counters_needed(int N);
+int gemm_row_blocks(int N, int K, int n, int epilogue);  // grid.x of the launch (size of argmax_partial)
 cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s);
 cudaError_t gemm_init();  // sets the dynamic shared memory limits once per process/device
+cudaError_t launch_argmax_finish(const float2* partial, int row_blocks, int n, int32_t* next, cudaStream_t s);
 
 // ---- paged decode attention -------------------------------------------------------
 struct AttnPlan {   // filled on the host from the request lengths
@@ -60,7 +79,9 @@ struct AttnArgs {
   int n_work, n, nq, nkv, max_blocks;
   float* part_acc;  // [slots][nq][128]
   float* part_ml;   // [slots][nq][2]
-  uint16_t* out;    // [n][nq][128]
+  uint16_t* out;    // plain [n][nq][128], or NULL
+  uint16_t* out_xp; // fragment-ordered operand [16][nq*128] of the O projection, or NULL
+  float* out_xs;    // its group sums [nq*2][16]
 };
 cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s);
@@ -85,8 +106,9 @@ cudaError_t launch_rope_append(const RopeArgs& a, cudaStream_t s);
 // ---- small kernels ----------------------------------------------------------------
 cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,
                          const int32_t* tokens, int n, uint16_t* x, cudaStream_t s);
+// y (plain, optional) and/or the fragment-ordered operand (yp, ys) of the next GEMM.
 cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int n, int H, uint16_t* y,
-                           cudaStream_t s);
+                           uint16_t* yp, float* ys, cudaStream_t s);
 cudaError_t launch_argmax(const float* logits, int n, int vocab, int32_t* next, cudaStream_t s);
 cudaError_t launch_dequant(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int N, int K,
                            float* out, cudaStream_t s);

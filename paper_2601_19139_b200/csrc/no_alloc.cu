@@ -21,7 +21,9 @@ namespace {
 
 constexpr size_t kCounterBytes = 16 * 1024;          // 4096 row-block counters
 constexpr size_t kPartialBytes = 8ull << 20;         // split-K partial sums
-constexpr size_t kScratchBytes = kCounterBytes + kPartialBytes;
+constexpr int kMaxK = 16384;                         // widest input the operand buffers hold
+constexpr size_t kOperandBytes = (size_t)16 * kMaxK * 2 + (size_t)(kMaxK / 64) * 16 * 4;  // operand + group sums
+constexpr size_t kScratchBytes = kCounterBytes + kPartialBytes + kOperandBytes;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
@@ -46,9 +48,9 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
   if (n < 0 || n > kMaxBatch || N < 1 || K < 256 || K % 256 || x_stride % 8 || prologue < 0 || prologue > 1 ||
       epilogue < 0 || epilogue > 2)
     return q4d_internal_fail(Q4D_ERR_INVALID_ARG, "q4_gemm_noalloc: bad shape (K must be a multiple of 256, n <= 16)");
-  const size_t need = gemm_partial_bytes(N, K);
+  const size_t need = gemm_partial_bytes(N, K, epilogue);
   const size_t need_counters = (size_t)gemm_counters_needed(N) * sizeof(int);
-  if (need > kPartialBytes || need_counters > kCounterBytes) {
+  if (need > kPartialBytes || need_counters > kCounterBytes || K > kMaxK) {
     snprintf(g_noalloc_error, sizeof g_noalloc_error,
              "q4_gemm_noalloc: a %d x %d projection needs %zu bytes of split-K scratch, the built-in array holds %zu; "
              "use q4d_q4_gemm with caller-provided scratch",
@@ -75,9 +77,15 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
   // The counters must be zero when the kernel starts; whatever an earlier call left is cleared here.
   e = cudaMemsetAsync(base, 0, need_counters, s);
   if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: clearing the counters failed");
+  // the activations are first rearranged into the order the GEMM reads them in, inside the same array
+  uint16_t* xp = reinterpret_cast<uint16_t*>(base + kCounterBytes + kPartialBytes);
+  float* xs = reinterpret_cast<float*>(base + kCounterBytes + kPartialBytes + (size_t)16 * kMaxK * 2);
+  e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, s);
+  if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: operand rearrangement failed");
   GemmArgs a;
-  a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.x = x, a.x_stride = x_stride, a.n = n;
-  a.prologue = prologue, a.epilogue = epilogue, a.out = out, a.out_stride = out_stride;
+  a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;
+  a.epilogue = epilogue, a.out = out, a.out_stride = out_stride;
+  a.out_xp = nullptr, a.out_xs = nullptr, a.argmax_partial = nullptr;
   a.counters = reinterpret_cast<int*>(base), a.counters_len = (int)(kCounterBytes / sizeof(int));
   a.partial = reinterpret_cast<float*>(base + kCounterBytes), a.partial_bytes = kPartialBytes;
   e = launch_q4_gemm(a, s);

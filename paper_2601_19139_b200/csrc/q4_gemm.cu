@@ -10,16 +10,21 @@
 // no dequantised weight is ever rounded to bf16; scale and bias are applied to
 // the fp32 group sums.
 //
-// Layout of the work.  A CTA of 8 warps owns 8*16*MT consecutive output rows
-// and one K-slice; each warp owns 16*MT rows and streams their packed codes,
-// scales and biases through a private cp.async ring in shared memory, 256 input
-// features (one "quad" of four groups, 128 B per row) per stage.  The
-// activation slice is staged once per CTA in shared memory in the element
-// order the MMA fragments need.  Split-K partial sums go to a scratch buffer;
-// the last CTA to arrive for a row block adds them in split order (so the
-// result does not depend on arrival order) and applies the epilogue.
+// Layout of the work.  A CTA of 8 warps owns 8*16*MT output rows and one
+// K-slice; each warp owns 16*MT rows and streams their packed codes, scales and
+// biases through a private cp.async ring in shared memory, 256 input features
+// (one "quad" of four groups, 128 B per row) per stage.  The activations arrive
+// already in MMA fragment order with their group sums (see common.cuh) and are
+// copied to shared memory asynchronously.  The weight stream does not depend on
+// the preceding kernel, so it is started before the grid dependency is awaited.
+// Split-K partial sums go to a scratch buffer; the last CTA to arrive for a row
+// block adds them in split order (the result does not depend on arrival order)
+// and applies the epilogue from a shared-memory tile.
+#include <stdlib.h>
+
 #include "common.cuh"
 #include "kernels.h"
+#include "launch.h"
 
 namespace q4d {
 
@@ -29,21 +34,24 @@ constexpr int kThreads = 256;
 constexpr int kWarps = 8;
 constexpr int kRowStride = 160;  // bytes per row per stage in smem: 128 data + 32 pad (conflict-free 8-byte reads)
 constexpr int kSbBytes = 16;     // per row per stage: 4 scales + 4 biases (bf16)
-constexpr int kStages = 3;
-constexpr int kMaxQuadsPerSlice = 8;  // K-slice <= 2048
+constexpr int kMaxQuadsPerSlice = 4;  // K-slice <= 1024
 
 struct GemmParams {
   const uint32_t* qw;
   const uint16_t* scales;
   const uint16_t* biases;
-  const uint16_t* x;
+  const uint16_t* xp;
+  const float* xs;
   void* out;
+  uint16_t* out_xp;
+  float* out_xs;
+  float2* argmax_partial;
   float* partial;
   int* counters;
-  int N, K, n, x_stride, out_stride;
+  int N, K, n, out_stride;
   int ks;      // nominal K-slice (multiple of 256)
   int splits;  // gridDim.y
-  int prologue, epilogue;
+  int epilogue;
 };
 
 // Four bf16x2 registers {code j, code j+4}, j = 0..3, as exact integers, from one packed word.
@@ -72,40 +80,53 @@ __device__ __forceinline__ void store_out(const GemmParams& p, int row, int req,
   }
 }
 
-template <int MT, int NT>
-__global__ void __launch_bounds__(kThreads, (MT == 1 && NT == 1) ? 2 : 1) q4_gemm_kernel(const GemmParams p) {
-  constexpr int R = 16 * MT;  // rows per warp
-  constexpr int NP = 8 * NT;  // padded request count
+template <int MT, int NT, int STAGES>
+__global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(const GemmParams p) {
+  constexpr int R = 16 * MT;        // rows per warp
+  constexpr int NP = 8 * NT;        // padded request count
+  constexpr int kRows = kWarps * R; // rows per CTA
   constexpr int kStage = R * (kRowStride + kSbBytes);
+  constexpr int kTs = NP + 1;       // row stride of the final tile (floats)
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ int s_is_last;
 
+  grid_launch_dependents();
+
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-  const int row_block = blockIdx.x * (kWarps * R);
-  const int warp_row0 = row_block + warp * R;
+  const bool silu = p.epilogue == EPI_SILU_PACK;
+  const int half_n = p.N >> 1;  // silu: rows [0, half_n) are gate rows, [half_n, N) up rows
+  // local row of the CTA -> row of the tensor.  With the SiLU epilogue the first half of the CTA's rows are
+  // gate rows and the second half the matching up rows, so that one CTA ends up with both.
+  auto global_row = [&](int lrow) -> int {
+    if (!silu) return blockIdx.x * kRows + lrow;
+    return lrow < kRows / 2 ? blockIdx.x * (kRows / 2) + lrow : half_n + blockIdx.x * (kRows / 2) + (lrow - kRows / 2);
+  };
+  const int row_limit_first = silu ? half_n : p.N;  // rows of the first half must stay below this
+  const int warp_row0 = global_row(warp * R);
+  const int warp_limit = (silu && warp * R >= kRows / 2) ? p.N : row_limit_first;
   const int k0 = blockIdx.y * p.ks;
   const int kend = min(p.K, k0 + p.ks);
   const int kslice = kend - k0;
   const int nquads = kslice >> 8;
   const int b_stride = p.ks * 2 + 16;  // bytes per request row of the staged activations
 
-  unsigned char* ring = smem + warp * (kStages * kStage);
-  unsigned char* sB = smem + kWarps * kStages * kStage;
+  unsigned char* ring = smem + warp * (STAGES * kStage);
+  unsigned char* sB = smem + kWarps * STAGES * kStage;
   float* sX = reinterpret_cast<float*>(sB + NP * b_stride);  // [group][NP]
 
   auto issue_stage = [&](int qd) {
-    unsigned char* stg = ring + (qd % kStages) * kStage;
+    unsigned char* stg = ring + (qd % STAGES) * kStage;
     const int kq = k0 + qd * 256;
 #pragma unroll
     for (int i = 0; i < R / 4; ++i) {
       const int r = i * 4 + (lane >> 3);
-      const int grow = min(warp_row0 + r, p.N - 1);
+      const int grow = min(warp_row0 + r, warp_limit - 1);
       const unsigned char* src =
           reinterpret_cast<const unsigned char*>(p.qw + (size_t)grow * (p.K >> 3) + (kq >> 3)) + (lane & 7) * 16;
       cp_async16(stg + r * kRowStride + (lane & 7) * 16, src);
     }
     for (int r = lane; r < R; r += 32) {
-      const int grow = min(warp_row0 + r, p.N - 1);
+      const int grow = min(warp_row0 + r, warp_limit - 1);
       const size_t off = (size_t)grow * (p.K >> 6) + (kq >> 6);
       cp_async8(stg + R * kRowStride + r * kSbBytes, p.scales + off);
       cp_async8(stg + R * kRowStride + r * kSbBytes + 8, p.biases + off);
@@ -114,50 +135,27 @@ __global__ void __launch_bounds__(kThreads, (MT == 1 && NT == 1) ? 2 : 1) q4_gem
 
   // Weights do not depend on the preceding kernel: start streaming them before waiting for it.
 #pragma unroll
-  for (int s = 0; s < kStages - 1; ++s) {
+  for (int s = 0; s < STAGES - 1; ++s) {
     if (s < nquads) issue_stage(s);
     cp_async_commit();
   }
 
   grid_dependency_wait();
 
-  // Stage the activation slice: permute each 8-element chunk to {0,4,1,5,2,6,3,7} so that a lane's
-  // 16 elements of a group are its B fragments of the four k-steps, and form the fp32 group sums.
+  // Activations (already in fragment order) and their group sums: straight copies.
   {
     const int cpr = kslice >> 3;  // 16-byte chunks per request row
-    const int total = NP * cpr;   // multiple of 256
-    for (int c = threadIdx.x; c < total; c += kThreads) {
+    for (int c = threadIdx.x; c < NP * cpr; c += kThreads) {
       const int r = c / cpr, kc = c - r * cpr;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < p.n) {
-        const uint16_t* src = p.x + (size_t)r * p.x_stride + k0 + kc * 8;
-        v = *reinterpret_cast<const uint4*>(src);
-        if (p.prologue == PRO_SILU_MUL) {
-          const uint4 u = *reinterpret_cast<const uint4*>(src + p.K);
-          uint32_t gw[4] = {v.x, v.y, v.z, v.w}, uw[4] = {u.x, u.y, u.z, u.w}, hw[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float g0 = bf16_lo(gw[i]), g1 = bf16_hi(gw[i]);
-            const float h0 = (g0 / (1.0f + expf(-g0))) * bf16_lo(uw[i]);
-            const float h1 = (g1 / (1.0f + expf(-g1))) * bf16_hi(uw[i]);
-            hw[i] = pack_bf16x2(h0, h1);
-          }
-          v = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-        }
-      }
-      float sum = ((bf16_lo(v.x) + bf16_hi(v.x)) + (bf16_lo(v.y) + bf16_hi(v.y))) +
-                  ((bf16_lo(v.z) + bf16_hi(v.z)) + (bf16_lo(v.w) + bf16_hi(v.w)));
-      sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-      sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-      uint4 o;
-      o.x = __byte_perm(v.x, v.z, 0x5410);
-      o.y = __byte_perm(v.x, v.z, 0x7632);
-      o.z = __byte_perm(v.y, v.w, 0x5410);
-      o.w = __byte_perm(v.y, v.w, 0x7632);
-      *reinterpret_cast<uint4*>(sB + r * b_stride + kc * 16) = o;
-      if ((kc & 7) == 0) sX[(kc >> 3) * NP + r] = sum;
+      cp_async16(sB + r * b_stride + kc * 16, p.xp + (size_t)r * p.K + k0 + kc * 8);
     }
+    const int groups = kslice >> 6;
+    for (int c = threadIdx.x; c < groups * (NP / 4); c += kThreads) {
+      const int gq = c / (NP / 4), q4 = c - gq * (NP / 4);
+      cp_async16(sX + gq * NP + q4 * 4, p.xs + (size_t)((k0 >> 6) + gq) * 16 + q4 * 4);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
   }
   __syncthreads();
 
@@ -170,11 +168,11 @@ __global__ void __launch_bounds__(kThreads, (MT == 1 && NT == 1) ? 2 : 1) q4_gem
       for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0f;
 
   for (int qd = 0; qd < nquads; ++qd) {
-    if (qd + kStages - 1 < nquads) issue_stage(qd + kStages - 1);
+    if (qd + STAGES - 1 < nquads) issue_stage(qd + STAGES - 1);
     cp_async_commit();
-    cp_async_wait<kStages - 1>();
+    cp_async_wait<STAGES - 1>();
     __syncwarp();
-    const unsigned char* stg = ring + (qd % kStages) * kStage;
+    const unsigned char* stg = ring + (qd % STAGES) * kStage;
 
     uint2 sc[MT][2], bi[MT][2];
 #pragma unroll
@@ -226,74 +224,139 @@ __global__ void __launch_bounds__(kThreads, (MT == 1 && NT == 1) ? 2 : 1) q4_gem
     __syncwarp();
   }
   cp_async_wait<0>();
+  __syncthreads();  // every warp is done with its ring: the final tile may overlay them
 
+  float* sT = reinterpret_cast<float*>(smem);  // [kRows][kTs]
   if (p.splits == 1) {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int row = warp_row0 + mt * 16 + g + (c >> 1) * 8;
-          const int req = nt * 8 + 2 * t + (c & 1);
-          if (row < p.N && req < p.n) store_out(p, row, req, acc[mt][nt][c]);
-        }
-    return;
-  }
-
-  // Split-K: publish this CTA's partial sums, then the last CTA of the row block reduces them.
-  const int n_pad = gridDim.x * (kWarps * R);
-  {
-    float* part = p.partial + (size_t)blockIdx.y * n_pad * NP;
+        for (int c = 0; c < 4; ++c)
+          sT[(warp * R + mt * 16 + g + (c >> 1) * 8) * kTs + nt * 8 + 2 * t + (c & 1)] = acc[mt][nt][c];
+  } else {
+    // Split-K: publish this CTA's partial sums, then the last CTA of the row block reduces them.
+    const size_t tile = (size_t)kRows * NP;
+    float* part = p.partial + ((size_t)blockIdx.y * gridDim.x + blockIdx.x) * tile;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const int row = warp_row0 + mt * 16 + g + h * 8;
-          *reinterpret_cast<float2*>(part + (size_t)row * NP + nt * 8 + 2 * t) =
+        for (int h = 0; h < 2; ++h)
+          *reinterpret_cast<float2*>(part + (size_t)(warp * R + mt * 16 + g + h * 8) * NP + nt * 8 + 2 * t) =
               make_float2(acc[mt][nt][2 * h], acc[mt][nt][2 * h + 1]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int prev = atomicAdd(p.counters + blockIdx.x, 1);
+      s_is_last = (prev == p.splits - 1);
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    __threadfence();
+    for (int idx = threadIdx.x; idx < kRows * NP / 4; idx += kThreads) {
+      const int lrow = idx / (NP / 4), q4 = idx - lrow * (NP / 4);
+      float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      for (int s = 0; s < p.splits; ++s) {
+        const float4 a = __ldcg(reinterpret_cast<const float4*>(p.partial + ((size_t)s * gridDim.x + blockIdx.x) * tile +
+                                                               (size_t)lrow * NP + q4 * 4));
+        v.x += a.x, v.y += a.y, v.z += a.z, v.w += a.w;
+      }
+      float* d = sT + lrow * kTs + q4 * 4;
+      d[0] = v.x, d[1] = v.y, d[2] = v.z, d[3] = v.w;
+    }
+    if (threadIdx.x == 0) p.counters[blockIdx.x] = 0;
+  }
+  __syncthreads();
+
+  if (silu) {
+    // h = bf16(silu(bf16(gate)) * bf16(up)) for the CTA's kRows/2 columns, as the next GEMM's operand.
+    constexpr int kCh = kRows / 16;  // chunks of 8 columns
+    const int idx = threadIdx.x;
+    if (idx < kCh * NP) {
+      const int c = idx % kCh, req = idx / kCh;
+      uint32_t hw[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float hv[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const int col = c * 8 + 2 * i + j;
+          const float gt = bf16_to_f32(f32_to_bf16(sT[col * kTs + req]));
+          const float up = bf16_to_f32(f32_to_bf16(sT[(kRows / 2 + col) * kTs + req]));
+          hv[j] = (gt / (1.0f + expf(-gt))) * up;
         }
+        hw[i] = pack_bf16x2(hv[0], hv[1]);
+      }
+      const uint4 v = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+      const float gsum = group_sum_8lanes(chunk_sum(v));
+      const int col0 = blockIdx.x * (kRows / 2) + c * 8;
+      if (col0 < half_n && req < p.n) {
+        *reinterpret_cast<uint4*>(p.out_xp + (size_t)req * half_n + col0) = permute_chunk(v);
+        if ((c & 7) == 0) p.out_xs[(size_t)(col0 >> 6) * 16 + req] = gsum;
+      }
+    }
+    return;
   }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int prev = atomicAdd(p.counters + blockIdx.x, 1);
-    s_is_last = (prev == p.splits - 1);
-  }
-  __syncthreads();
-  if (!s_is_last) return;
-  __threadfence();
-  constexpr int kRows = kWarps * R;
+
   for (int idx = threadIdx.x; idx < kRows * NP; idx += kThreads) {
-    const int req = idx / kRows, row = row_block + (idx - req * kRows);
-    if (row >= p.N || req >= p.n) continue;
-    float v = 0.0f;
-    for (int s = 0; s < p.splits; ++s) v += __ldcg(p.partial + ((size_t)s * n_pad + row) * NP + req);
-    store_out(p, row, req, v);
+    const int req = idx / kRows, lrow = idx - req * kRows;
+    const int row = blockIdx.x * kRows + lrow;
+    if (row < p.N && req < p.n) store_out(p, row, req, sT[lrow * kTs + req]);
   }
-  if (threadIdx.x == 0) p.counters[blockIdx.x] = 0;
+  if (p.epilogue == EPI_F32 && p.argmax_partial) {
+    // Per request: the largest value of this row block and its row (lowest row among equals).
+    for (int req = warp; req < NP; req += kWarps) {
+      float best = -INFINITY;
+      int bidx = 0x7fffffff;
+      for (int lrow = lane; lrow < kRows; lrow += 32) {
+        const int row = blockIdx.x * kRows + lrow;
+        const float v = sT[lrow * kTs + req];
+        if (row < p.N && (v > best || (v == best && row < bidx))) best = v, bidx = row;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bidx, o);
+        if (ov > best || (ov == best && oi < bidx)) best = ov, bidx = oi;
+      }
+      if (lane == 0 && req < p.n) p.argmax_partial[(size_t)blockIdx.x * 16 + req] = make_float2(best, __int_as_float(bidx));
+    }
+  }
 }
 
-template <int MT, int NT>
+template <int MT, int NT, int STAGES>
 size_t smem_bytes(int ks) {
-  return (size_t)kWarps * kStages * (16 * MT) * (kRowStride + kSbBytes) + (size_t)(8 * NT) * (ks * 2 + 16) +
+  return (size_t)kWarps * STAGES * (16 * MT) * (kRowStride + kSbBytes) + (size_t)(8 * NT) * (ks * 2 + 16) +
          (size_t)(ks / 64) * (8 * NT) * sizeof(float);
 }
 
 struct Tiling {
-  int mt, nt, rows_cta, rowblocks, qps, splits;
+  int cfg;  // 0: <1,1,4>  1: <2,2,4>  2: <1,2,3>
+  int nt, rows_cta, rowblocks, qps, splits;
 };
 
-Tiling choose_tiling(int N, int K, int n, int sm_count) {
+int g_sm_count = 0;
+int g_force_cfg = -1;  // debugging aid: environment variable Q4D_GEMM_CFG forces the n > 8 configuration
+
+Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count) {
   Tiling t;
-  t.nt = n > 8 ? 2 : 1;
-  t.mt = t.nt == 2 ? 2 : 1;
-  t.rows_cta = kWarps * 16 * t.mt;
-  t.rowblocks = (N + t.rows_cta - 1) / t.rows_cta;
+  const int rows_logical = epilogue == EPI_SILU_PACK ? N / 2 : N;  // rows that index row blocks
   const int quads = K / 256;
-  const int wave = sm_count * ((t.mt == 1 && t.nt == 1) ? 2 : 1);
+  if (n <= 8) {
+    t.cfg = 0, t.nt = 1, t.rows_cta = 128;
+  } else {
+    // 256-row CTAs (one per SM) when they fill the machine, else 128-row CTAs (two per SM)
+    const int rb256 = (rows_logical + 127) / 128 / (epilogue == EPI_SILU_PACK ? 1 : 2);
+    t.cfg = (long long)rb256 * quads >= sm_count ? 1 : 2;
+    if (g_force_cfg == 1 || g_force_cfg == 2) t.cfg = g_force_cfg;
+    t.nt = 2, t.rows_cta = t.cfg == 1 ? 256 : 128;
+  }
+  const int rows_per_block = epilogue == EPI_SILU_PACK ? t.rows_cta / 2 : t.rows_cta;
+  t.rowblocks = (rows_logical + rows_per_block - 1) / rows_per_block;
+  const int wave = sm_count * (t.cfg == 1 ? 1 : 2);
   int qps = 1;
   for (int c = (quads < kMaxQuadsPerSlice ? quads : kMaxQuadsPerSlice); c >= 1; --c) {
     if (quads % c) continue;
@@ -307,30 +370,72 @@ Tiling choose_tiling(int N, int K, int n, int sm_count) {
   return t;
 }
 
-int g_sm_count = 0;
+size_t tiling_partial_bytes(const Tiling& t) {
+  return t.splits > 1 ? (size_t)t.splits * t.rowblocks * t.rows_cta * (8 * t.nt) * sizeof(float) : 0;
+}
+
+int sm_count_or_default() {
+  if (g_sm_count == 0) {
+    if (gemm_init() != cudaSuccess) {
+      (void)cudaGetLastError();
+      return 148;  // sizing only: no device in this process
+    }
+  }
+  return g_sm_count;
+}
+
+// next[r] = the best of the row-block partial results, lowest index among equals.
+__global__ void __launch_bounds__(256) argmax_finish_kernel(const float2* partial, int row_blocks, int32_t* next) {
+  __shared__ float sv[8];
+  __shared__ int si[8];
+  grid_launch_dependents();
+  grid_dependency_wait();
+  const int req = blockIdx.x;
+  float best = -INFINITY;
+  int bidx = 0x7fffffff;
+  for (int b = threadIdx.x; b < row_blocks; b += blockDim.x) {
+    const float2 v = partial[(size_t)b * 16 + req];
+    const int i = __float_as_int(v.y);
+    if (v.x > best || (v.x == best && i < bidx)) best = v.x, bidx = i;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bidx, o);
+    if (ov > best || (ov == best && oi < bidx)) best = ov, bidx = oi;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) sv[warp] = best, si[warp] = bidx;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w)
+      if (sv[w] > best || (sv[w] == best && si[w] < bidx)) best = sv[w], bidx = si[w];
+    next[req] = bidx == 0x7fffffff ? 0 : bidx;
+  }
+}
 
 }  // namespace
 
-size_t gemm_partial_bytes(int N, int K) {
-  int sms = g_sm_count;
-  if (sms == 0) {
-    if (gemm_init() == cudaSuccess) {
-      sms = g_sm_count;
-    } else {
-      (void)cudaGetLastError();
-      sms = 148;  // sizing only: no device in this process
-    }
-  }
+size_t gemm_partial_bytes(int N, int K, int epilogue) {
+  const int sms = sm_count_or_default();
   size_t need = 0;
-  for (int n = 8; n <= 16; n += 8) {  // the two tilings: up to 8 requests, 9..16 requests
-    const Tiling t = choose_tiling(N, K, n, sms);
-    const size_t b = t.splits > 1 ? (size_t)t.splits * t.rowblocks * t.rows_cta * (8 * t.nt) * sizeof(float) : 0;
-    if (b > need) need = b;
+  for (int n = 8; n <= 16; n += 8) {  // the tilings: up to 8 requests, 9..16 requests (either CTA size)
+    for (int force = 1; force <= 2; ++force) {
+      const int saved = g_force_cfg;
+      g_force_cfg = n > 8 ? force : saved;
+      const size_t b = tiling_partial_bytes(choose_tiling(N, K, n, epilogue, sms));
+      g_force_cfg = saved;
+      if (b > need) need = b;
+    }
   }
   return need;
 }
 
-int gemm_counters_needed(int N) { return (N + 127) / 128 + 1; }
+int gemm_counters_needed(int N) { return (N + 63) / 64 + 1; }
+
+int gemm_row_blocks(int N, int K, int n, int epilogue) {
+  return choose_tiling(N, K, n, epilogue, sm_count_or_default()).rowblocks;
+}
 
 cudaError_t gemm_init() {
   int dev = 0;
@@ -341,10 +446,13 @@ cudaError_t gemm_init() {
   if (e != cudaSuccess) return e;
   // 227 KB is the per-CTA limit for static + dynamic shared memory; leave room for the static part.
   const int big = 227 * 1024 - 1024;
-  e = cudaFuncSetAttribute(q4_gemm_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, big / 2 - 1024);
+  e = cudaFuncSetAttribute(q4_gemm_kernel<1, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big / 2 - 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_gemm_kernel<2, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big / 2 - 1024);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(q4_gemm_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e != cudaSuccess) return e;
+  if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   g_sm_count = sms;
   return cudaSuccess;
 }
@@ -355,24 +463,33 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
   }
   if (a.n <= 0) return cudaSuccess;
-  if (a.N <= 0 || a.K <= 0 || (a.K % 256) || a.n > kMaxBatch || (a.x_stride % 8)) return cudaErrorInvalidValue;
-  const Tiling t = choose_tiling(a.N, a.K, a.n, g_sm_count);
+  if (a.N <= 0 || a.K <= 0 || (a.K % 256) || a.n > kMaxBatch) return cudaErrorInvalidValue;
+  if (a.epilogue == EPI_SILU_PACK && ((a.N % 16) || !a.out_xp || !a.out_xs)) return cudaErrorInvalidValue;
+  const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count);
   GemmParams p;
-  p.qw = a.qw, p.scales = a.scales, p.biases = a.biases, p.x = a.x, p.out = a.out;
+  p.qw = a.qw, p.scales = a.scales, p.biases = a.biases, p.xp = a.xp, p.xs = a.xs, p.out = a.out;
+  p.out_xp = a.out_xp, p.out_xs = a.out_xs, p.argmax_partial = a.argmax_partial;
   p.partial = a.partial, p.counters = a.counters;
-  p.N = a.N, p.K = a.K, p.n = a.n, p.x_stride = a.x_stride, p.out_stride = a.out_stride;
-  p.ks = t.qps * 256, p.splits = t.splits, p.prologue = a.prologue, p.epilogue = a.epilogue;
+  p.N = a.N, p.K = a.K, p.n = a.n, p.out_stride = a.out_stride;
+  p.ks = t.qps * 256, p.splits = t.splits, p.epilogue = a.epilogue;
   if (t.splits > 1) {
-    const size_t need = (size_t)t.splits * t.rowblocks * t.rows_cta * (8 * t.nt) * sizeof(float);
-    if (!a.partial || !a.counters || need > a.partial_bytes || t.rowblocks > a.counters_len)
+    if (!a.partial || !a.counters || tiling_partial_bytes(t) > a.partial_bytes || t.rowblocks > a.counters_len)
       return cudaErrorInvalidValue;
   }
   const dim3 grid(t.rowblocks, t.splits), block(kThreads);
-  if (t.mt == 1 && t.nt == 1)
-    q4_gemm_kernel<1, 1><<<grid, block, smem_bytes<1, 1>(p.ks), s>>>(p);
-  else
-    q4_gemm_kernel<2, 2><<<grid, block, smem_bytes<2, 2>(p.ks), s>>>(p);
-  return cudaGetLastError();
+  switch (t.cfg) {
+    case 0:
+      return launch_kernel(q4_gemm_kernel<1, 1, 4>, grid, block, smem_bytes<1, 1, 4>(p.ks), s, p);
+    case 1:
+      return launch_kernel(q4_gemm_kernel<2, 2, 4>, grid, block, smem_bytes<2, 2, 4>(p.ks), s, p);
+    default:
+      return launch_kernel(q4_gemm_kernel<1, 2, 3>, grid, block, smem_bytes<1, 2, 3>(p.ks), s, p);
+  }
+}
+
+cudaError_t launch_argmax_finish(const float2* partial, int row_blocks, int n, int32_t* next, cudaStream_t s) {
+  if (n <= 0) return cudaSuccess;
+  return launch_kernel(argmax_finish_kernel, dim3(n), dim3(256), 0, s, partial, row_blocks, next);
 }
 
 }  // namespace q4d

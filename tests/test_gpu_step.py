@@ -90,8 +90,10 @@ def _run_steps(q4d, sc, steps):
     return agree, total, worst_max, worst_rms
 
 
-def _layerwise(q4d, sc):
+def _layerwise(q4d, sc, production=True):
     """Each layer on the GPU from the oracle's input to that layer; then the head from the oracle's final state.
+    production=True runs the layer through q4d_debug_run_layers (the step's own launch sequence); otherwise the
+    layer is composed from the single-operation entry points.
     Returns (worst per-layer (max, rms, mismatch), logit max error, tokens equal, n)."""
     shape, lens = sc.shape, sc.lens
     n = len(lens)
@@ -103,9 +105,19 @@ def _layerwise(q4d, sc):
     x0 = q4d.embed(sc.weights["embed"], torch.from_numpy(sc.tokens).cuda())
     assert np.array_equal(bits(x0), taps[0])
     worst = [0.0, 0.0, 0.0]
+    model = pool = None
+    ids = np.arange(n, dtype=np.int64)
+    if production:
+        model = q4d.Model(shape, sc.weights)
+        pool = q4d.KVPool(model, sc.pool)
+        for r in range(n):
+            pool.request_admit(r, lens[r])
     for l in range(shape.n_layers):
         x = from_bits(taps[l])
-        gpu_layer(q4d, shape, sc.weights, l, x, sc.pool, lens, dlens, dbt, oracle_pool=o_pool, bt=bt)
+        if production:
+            x = q4d.debug_run_layers(model, pool, ids, bt, l, l + 1, x)
+        else:
+            gpu_layer(q4d, shape, sc.weights, l, x, sc.pool, lens, dlens, dbt, oracle_pool=o_pool, bt=bt)
         torch.cuda.synchronize()
         e = rel_err(bits(x), taps[l + 1])
         worst = [max(a, b) for a, b in zip(worst, e)]
@@ -113,6 +125,9 @@ def _layerwise(q4d, sc):
         # fraction of a step
         assert_bf16_close(bits(x), taps[l + 1], max_ulp=10, max_mismatch_frac=0.7, what=f"layer {l} output")
         assert e[1] <= 6e-3, (l, e)
+    if production:
+        pool.close()
+        model.close()
     y = q4d.rmsnorm(from_bits(taps[-1]), sc.weights["final_norm"], shape.rms_eps)
     lg = q4d.q4_gemm(sc.weights["lm_head"], y, n, epilogue=2)
     nxt = q4d.argmax(lg).cpu().numpy()
@@ -145,10 +160,11 @@ def test_toy_whole_steps_match_oracle(q4d, shape, lens):
     assert agree >= total - max(1, total // 50), (agree, total)
 
 
+@pytest.mark.parametrize("production", [True, False], ids=["step-path", "composed-ops"])
 @pytest.mark.parametrize("shape,lens", TOYS, ids=[t[0].name for t in TOYS])
-def test_toy_layers_match_oracle_teacher_forced(q4d, shape, lens):
+def test_toy_layers_match_oracle_teacher_forced(q4d, shape, lens, production):
     sc = Scenario(shape, lens, seed=4)
-    _, emax, same, n = _layerwise(q4d, sc)
+    _, emax, same, n = _layerwise(q4d, sc, production)
     assert emax <= LOGIT_TOL and same == n
 
 
