@@ -229,16 +229,19 @@ __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs p) 
   float den = 0.0f;
   if (valid) {
     float M = -INFINITY;
-    for (int c = 0; c < nc; ++c) M = fmaxf(M, p.part_ml[((size_t)(s0 + c) * p.nq + a) * 2]);
+#pragma unroll 8
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(p.part_ml + ((size_t)(s0 + c) * p.nq + a) * 2));
+#pragma unroll 4
     for (int c = 0; c < nc; ++c) {
       const size_t qh = (size_t)(s0 + c) * p.nq + a;
-      const float e = exp2f(p.part_ml[qh * 2] - M);
-      const float4 u = *reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8);
-      const float4 v = *reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8 + 4);
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + qh * 2));
+      const float4 u = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8));
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8 + 4));
+      const float e = exp2f(ml.x - M);
       acc[0] = fmaf(e, u.x, acc[0]), acc[1] = fmaf(e, u.y, acc[1]), acc[2] = fmaf(e, u.z, acc[2]);
       acc[3] = fmaf(e, u.w, acc[3]), acc[4] = fmaf(e, v.x, acc[4]), acc[5] = fmaf(e, v.y, acc[5]);
       acc[6] = fmaf(e, v.z, acc[6]), acc[7] = fmaf(e, v.w, acc[7]);
-      den = fmaf(e, p.part_ml[qh * 2 + 1], den);
+      den = fmaf(e, ml.y, den);
     }
   } else {
     den = 1.0f;

@@ -6,9 +6,9 @@
 //         = sum_g scale[j][g] * (sum_{k in g} q[j][k] x[r][k]) + bias[j][g] * (sum_{k in g} x[r][k])
 //
 // The inner sums run on the tensor cores with the 4-bit codes converted to
-// exact bf16 integers (products code * x are exact, accumulation is fp32), so
-// no dequantised weight is ever rounded to bf16; scale and bias are applied to
-// the fp32 group sums.
+// exact bf16 integers 16 + q (products are exact, accumulation is fp32), so
+// no dequantised weight is ever rounded to bf16; scale and bias (less 16 * scale,
+// which removes the offset again) are applied to the fp32 group sums.
 //
 // Layout of the work.  A CTA of 8 warps owns 8*16*MT output rows and one
 // K-slice; each warp owns 16*MT rows and streams their packed codes, scales and
@@ -54,14 +54,15 @@ struct GemmParams {
   int epilogue;
 };
 
-// Four bf16x2 registers {code j, code j+4}, j = 0..3, as exact integers, from one packed word.
+// Four bf16x2 registers {16 + code j, 16 + code j+4}, j = 0..3, from one packed word: the code is placed in
+// mantissa bits 3..6 of bf16 16.0 (0x4180), where 16 + code is exact.  One shift and one logic op per register;
+// the constant 16 is taken out again through the group sums (16 * sum x is subtracted via the bias term).
 __device__ __forceinline__ void unpack_word(uint32_t w, uint32_t (&p)[4]) {
-  constexpr uint32_t kMask = 0x000F000Fu, kMagic = 0x43004300u;  // bf16 128.0 in both halves
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    uint32_t v = ((w >> (4 * j)) & kMask) | kMagic;  // 128 + code, exact
-    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(p[j]) : "r"(v), "r"(kMagic));
-  }
+  constexpr uint32_t kMask = 0x00780078u, kSixteen = 0x41804180u;
+  p[0] = ((w << 3) & kMask) | kSixteen;
+  p[1] = ((w >> 1) & kMask) | kSixteen;
+  p[2] = ((w >> 5) & kMask) | kSixteen;
+  p[3] = ((w >> 9) & kMask) | kSixteen;
 }
 
 __device__ __forceinline__ float bf16_at(const uint2& v, int i) {
@@ -205,8 +206,9 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
         unpack_word(wl.y, l1);
         unpack_word(wh.x, h0);
         unpack_word(wh.y, h1);
+        // sum (16 + q) x = 16 X + sum q x, so the bias that multiplies X becomes b - 16 s
         const float s_lo = bf16_at(sc[mt][0], gi), s_hi = bf16_at(sc[mt][1], gi);
-        const float b_lo = bf16_at(bi[mt][0], gi), b_hi = bf16_at(bi[mt][1], gi);
+        const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[mt][0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[mt][1], gi));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
           float pc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -350,7 +352,8 @@ Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count) {
   } else {
     // 256-row CTAs (one per SM) when they fill the machine, else 128-row CTAs (two per SM)
     const int rb256 = (rows_logical + 127) / 128 / (epilogue == EPI_SILU_PACK ? 1 : 2);
-    t.cfg = (long long)rb256 * quads >= sm_count ? 1 : 2;
+    (void)rb256;
+    t.cfg = 2;  // two 128-row CTAs per SM hide more latency than one 256-row CTA (measured)
     if (g_force_cfg == 1 || g_force_cfg == 2) t.cfg = g_force_cfg;
     t.nt = 2, t.rows_cta = t.cfg == 1 ? 256 : 128;
   }
