@@ -234,7 +234,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
  * every GPU holds from the moment the library is loaded until the process exits.  The call allocates
  * and frees nothing.
  *  - Projections whose split-K partial sums exceed the array, or with K > 16384, are refused with
- *    WORKSPACE_TOO_SMALL (for example a 151936 x 4096 LM head at batch 16); use q4d_q4_gemm then.
+ *    WORKSPACE_TOO_SMALL (for example a 69632 x 8192 projection); use q4d_q4_gemm then.
  *  - The first call on each device looks up the array's device address; make that first call
  *    outside any stream capture, with the device current.
  *  - Every call reuses the same array and finds in it what the previous call left; the counters are

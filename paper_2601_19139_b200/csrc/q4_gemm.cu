@@ -57,12 +57,17 @@ struct GemmParams {
 // Four bf16x2 registers {16 + code j, 16 + code j+4}, j = 0..3, from one packed word: the code is placed in
 // mantissa bits 3..6 of bf16 16.0 (0x4180), where 16 + code is exact.  One shift and one logic op per register;
 // the constant 16 is taken out again through the group sums (16 * sum x is subtracted via the bias term).
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {  // (a & b) | c in one LOP3
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 __device__ __forceinline__ void unpack_word(uint32_t w, uint32_t (&p)[4]) {
-  constexpr uint32_t kMask = 0x00780078u, kSixteen = 0x41804180u;
-  p[0] = ((w << 3) & kMask) | kSixteen;
-  p[1] = ((w >> 1) & kMask) | kSixteen;
-  p[2] = ((w >> 5) & kMask) | kSixteen;
-  p[3] = ((w >> 9) & kMask) | kSixteen;
+  const uint32_t kMask = 0x00780078u, kSixteen = 0x41804180u;
+  p[0] = and_or(w << 3, kMask, kSixteen);
+  p[1] = and_or(w >> 1, kMask, kSixteen);
+  p[2] = and_or(w >> 5, kMask, kSixteen);
+  p[3] = and_or(w >> 9, kMask, kSixteen);
 }
 
 __device__ __forceinline__ float bf16_at(const uint2& v, int i) {
@@ -211,8 +216,8 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
         const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[mt][0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[mt][1], gi));
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-          float pc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-          mma_bf16(pc, l0[0], h0[0], l0[1], h0[1], bf[nt][0].x, bf[nt][0].y);
+          float pc[4];
+          mma_bf16_first(pc, l0[0], h0[0], l0[1], h0[1], bf[nt][0].x, bf[nt][0].y);
           mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
           mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
           mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);

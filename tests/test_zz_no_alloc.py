@@ -31,7 +31,7 @@ def _x(n, K, seed):
 
 def test_noalloc_gemm_equals_the_scratch_taking_entry_point_twice_in_a_row(q4d):
     # outputs are allocated before the calls under test: the entry point itself must allocate nothing
-    cases = [(4096, 4096, 16, 2), (1024, 3072, 5, 0)]     # split-K in both; f32 then bf16 epilogue
+    cases = [(4096, 12288, 16, 2), (1024, 8192, 5, 0)]    # K > 4096: partial sums go through the array
     prepared = []
     for i, (N, K, n, epi) in enumerate(cases):
         w = gen.random_q4(N, K, "cuda", "noalloc", i)
@@ -57,7 +57,7 @@ def test_noalloc_gemm_equals_the_scratch_taking_entry_point_twice_in_a_row(q4d):
 
 
 def test_noalloc_gemm_refuses_shapes_beyond_its_array(q4d):
-    N, K, n = 151936, 4096, 16
+    N, K, n = 69632, 8192, 16                              # 2 x 69632 x 16 partial sums: more than 8 MiB
     w = gen.random_q4(N, K, "cuda", "noalloc-big")
     x = _x(n, K, 50)
     out = torch.zeros(n, N, dtype=torch.float32, device="cuda")
