@@ -339,9 +339,19 @@ AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, i
   if (chunk_tokens > 0) {
     chunk_tiles = (chunk_tokens + 15) / 16;
   } else {
-    // Largest chunk (up to 1024 tokens) that still yields about four CTAs per SM.
-    chunk_tiles = 64;
-    while (chunk_tiles > 4 && (total_tiles / chunk_tiles + n) * nkv < 4LL * sm_count) chunk_tiles >>= 1;
+    // One wave: two CTAs fit on an SM, so aim at 2 * sm_count items of equal size (a multiple of 4 tiles so
+    // that the four warps of a CTA get equal shares), at least 4 tiles and at most 64.
+    const long long slots = 2LL * sm_count;
+    long long ct = (total_tiles * nkv + slots - 1) / slots;
+    ct = (ct + 3) / 4 * 4;
+    chunk_tiles = (int)(ct < 4 ? 4 : (ct > 64 ? 64 : ct));
+    // requests add a ragged last chunk each: grow the chunk until the items fit the wave
+    for (;;) {
+      long long items = 0;
+      for (int r = 0; r < n; ++r) items += ((lens[r] + 1 + 15) / 16 + chunk_tiles - 1) / chunk_tiles;
+      if (items * nkv <= slots || chunk_tiles >= 64) break;
+      chunk_tiles += 4;
+    }
   }
   if (chunk_tiles < 1) chunk_tiles = 1;
   int w = 0;
