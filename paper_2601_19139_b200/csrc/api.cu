@@ -63,6 +63,8 @@ struct Workspace {
   // (normed hidden state, attention output, silu(gate)*up).
   size_t x, yp, ys, qkv, qbuf, ap, as, hp, hs, logits, next, amax, gemm_partial, gemm_partial_bytes, counters,
       part_acc, part_ml, meta, bytes;
+  // MoE: plain normed state, routing results, touched-expert list, per-slot expert activations and outputs
+  size_t yplain, m_idx, m_wgt, m_ints, m_hp, m_hs, m_o;
   int counters_len, amax_blocks;
 };
 
@@ -82,7 +84,9 @@ bool shape_supported(const q4d_shape& s, std::string* why) {
   if (s.n_experts == 0) {
     if (s.mlp_inter < 256 || s.mlp_inter % 256) return bad("mlp_inter must be a positive multiple of 256");
   } else {
-    return bad("MoE layers are not supported yet");
+    if (s.n_experts > 256 || s.top_k < 1 || s.top_k > 32 || s.top_k > s.n_experts) return bad("need 1 <= top_k <= min(32, n_experts), n_experts <= 256");
+    if (s.expert_inter < 256 || s.expert_inter % 256 || s.expert_inter > 2048) return bad("expert_inter must be a multiple of 256, at most 2048");
+    if (s.hidden > 2048) return bad("MoE layers need hidden <= 2048");
   }
   return true;
 }
@@ -105,8 +109,19 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   w.qbuf = take(B * qdim * 2);
   w.ap = take(B * qdim * 2);
   w.as = take((qdim / 64) * 16 * 4);
-  w.hp = take(B * (size_t)s.mlp_inter * 2);
-  w.hs = take((size_t)(s.mlp_inter / 64) * 16 * 4);
+  w.hp = take(B * (size_t)s.mlp_inter * 2 + 256);
+  w.hs = take((size_t)(s.mlp_inter / 64) * 16 * 4 + 256);
+  w.yplain = w.m_idx = w.m_wgt = w.m_ints = w.m_hp = w.m_hs = w.m_o = 0;
+  if (s.n_experts) {
+    const size_t E = s.n_experts;
+    w.yplain = take(B * s.hidden * 2);
+    w.m_idx = take(B * s.top_k * 4);
+    w.m_wgt = take(B * s.top_k * 4);
+    w.m_ints = take((3 * E + 2) * 4);  // flags[E], expert_ids[E], slot_of[E], counter, n_touched
+    w.m_hp = take(E * B * s.expert_inter * 2);
+    w.m_hs = take(E * (size_t)(s.expert_inter / 64) * 16 * 4);
+    w.m_o = take(E * B * s.hidden * 2);
+  }
   w.logits = take(B * (size_t)s.vocab * 4);
   w.next = take(B * 4);
   w.amax_blocks = (s.vocab + 127) / 128 + 1;
@@ -119,8 +134,10 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   };
   gemm(nqkv, s.hidden, EPI_BF16);
   gemm(s.hidden, s.n_q_heads * kHeadDim, EPI_RESIDUAL);
-  gemm(2 * s.mlp_inter, s.hidden, EPI_SILU_PACK);
-  gemm(s.hidden, s.mlp_inter, EPI_RESIDUAL);
+  if (!s.n_experts) {
+    gemm(2 * s.mlp_inter, s.hidden, EPI_SILU_PACK);
+    gemm(s.hidden, s.mlp_inter, EPI_RESIDUAL);
+  }
   gemm(s.vocab, s.hidden, EPI_F32);
   w.gemm_partial_bytes = pb;
   w.gemm_partial = take(pb);
@@ -355,11 +372,40 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
     Q4D_LAUNCH(Q4D_K_ATTN_MERGE, launch_attention_merge(aa, s));
     Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
-    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
-    GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
-    gu.out_xp = hp, gu.out_xs = hs;
-    Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
-    Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
+    if (sh.n_experts == 0) {
+      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+      GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
+      gu.out_xp = hp, gu.out_xs = hs;
+      Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
+      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
+    } else {
+      const int E = sh.n_experts, Ie = sh.expert_inter;
+      uint16_t* yplain = at<uint16_t>(m, m->lay.yplain);
+      int32_t* ints = at<int32_t>(m, m->lay.m_ints);
+      MoeRouteArgs mr;
+      mr.y = yplain, mr.router = lw.router, mr.H = H, mr.E = E, mr.top_k = sh.top_k, mr.norm = sh.norm_topk_prob;
+      mr.idx = at<int32_t>(m, m->lay.m_idx), mr.wgt = at<float>(m, m->lay.m_wgt);
+      mr.flags = ints, mr.expert_ids = ints + E, mr.slot_of = ints + 2 * E, mr.counter = ints + 3 * E;
+      mr.n_touched = ints + 3 * E + 1;
+      uint16_t* ehp = at<uint16_t>(m, m->lay.m_hp);
+      float* ehs = at<float>(m, m->lay.m_hs);
+      uint16_t* eo = at<uint16_t>(m, m->lay.m_o);
+      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, yplain, yp, ys, s));
+      Q4D_LAUNCH(Q4D_K_MOE_ROUTER, launch_moe_router(mr, n, s));
+      GemmArgs gu = gemm_args(m, lw.experts_gate_up, 2 * Ie, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
+      gu.out_xp = ehp, gu.out_xs = ehs;
+      gu.expert_ids = mr.expert_ids, gu.n_touched = mr.n_touched, gu.max_slots = E;
+      gu.out_slot_stride = (size_t)16 * Ie, gu.out_xs_slot_stride = (size_t)(Ie / 64) * 16;
+      Q4D_LAUNCH(Q4D_K_MOE_GATE_UP, launch_q4_gemm(gu, s));
+      GemmArgs dn = gemm_args(m, lw.experts_down, H, Ie, ehp, ehs, n, EPI_BF16, eo, H);
+      dn.expert_ids = mr.expert_ids, dn.n_touched = mr.n_touched, dn.max_slots = E;
+      dn.xp_slot_stride = (size_t)16 * Ie, dn.xs_slot_stride = (size_t)(Ie / 64) * 16;
+      dn.out_slot_stride = (size_t)16 * H;
+      Q4D_LAUNCH(Q4D_K_MOE_DOWN, launch_q4_gemm(dn, s));
+      MoeCombineArgs mc;
+      mc.x = x, mc.o = eo, mc.idx = mr.idx, mc.wgt = mr.wgt, mc.slot_of = mr.slot_of, mc.H = H, mc.top_k = sh.top_k;
+      Q4D_LAUNCH(Q4D_K_MOE_DOWN, launch_moe_combine(mc, n, s));
+    }
   }
   if (range) {
     cudaError_t ce = cudaMemcpyAsync(range->x_out, x, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
@@ -415,8 +461,10 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
     return fail(Q4D_ERR_INVALID_ARG, "model_create: missing tensor");
   for (int l = 0; l < shape->n_layers; ++l) {
     const q4d_layer_weights& lw = weights->layers[l];
-    if (!lw.attn_norm || !lw.mlp_norm || !qt_ok(lw.wqkv) || !qt_ok(lw.wo) || !qt_ok(lw.w_gate_up) ||
-        !qt_ok(lw.w_down) || (shape->qk_norm && (!lw.q_norm || !lw.k_norm)))
+    const bool mlp_ok = shape->n_experts ? (lw.router && qt_ok(lw.experts_gate_up) && qt_ok(lw.experts_down))
+                                         : (qt_ok(lw.w_gate_up) && qt_ok(lw.w_down));
+    if (!lw.attn_norm || !lw.mlp_norm || !qt_ok(lw.wqkv) || !qt_ok(lw.wo) || !mlp_ok ||
+        (shape->qk_norm && (!lw.q_norm || !lw.k_norm)))
       return fail(Q4D_ERR_INVALID_ARG, "model_create: layer %d has a missing tensor", l);
   }
   MetaLayout ml;
@@ -453,6 +501,8 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   }
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_next), kMaxBatch * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
+  if (e == cudaSuccess && shape->n_experts)
+    e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 2) * 4);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     q4d_model_destroy(m);

@@ -46,6 +46,12 @@ struct GemmArgs {
   size_t partial_bytes;
   int* counters;  // zero between launches
   int counters_len;
+  // grouped mode (MoE): one GEMM per slot of a device-side list of touched experts; the tensors hold
+  // `N` rows per expert, stacked.  NULL expert_ids = a single GEMM.
+  const int* expert_ids = nullptr;  // [max_slots]
+  const int* n_touched = nullptr;   // number of valid slots
+  int max_slots = 0;
+  size_t xp_slot_stride = 0, xs_slot_stride = 0, out_slot_stride = 0, out_xs_slot_stride = 0;  // elements
 };
 
 // Bytes of split-K scratch a GEMM of this shape may use (upper bound over batch sizes).
@@ -102,6 +108,30 @@ struct RopeArgs {
   uint16_t* q_out;
 };
 cudaError_t launch_rope_append(const RopeArgs& a, cudaStream_t s);
+
+// ---- mixture of experts ------------------------------------------------------------
+struct MoeRouteArgs {
+  const uint16_t* y;       // plain normed hidden state bf16 [n][H]
+  const uint16_t* router;  // bf16 [E][H]
+  int H, E, top_k, norm;
+  int32_t* idx;         // [16][top_k] selected experts, by decreasing logit
+  float* wgt;           // [16][top_k] their weights
+  int32_t* flags;       // [E], zero between launches
+  int32_t* counter;     // zero between launches
+  int32_t* expert_ids;  // [E] touched experts, ascending
+  int32_t* slot_of;     // [E] position of an expert in expert_ids
+  int32_t* n_touched;
+};
+struct MoeCombineArgs {
+  uint16_t* x;        // residual stream bf16 [n][H], updated in place
+  const uint16_t* o;  // expert outputs bf16 [slot][16][H]
+  const int32_t* idx;
+  const float* wgt;
+  const int32_t* slot_of;
+  int H, top_k;
+};
+cudaError_t launch_moe_router(const MoeRouteArgs& a, int n, cudaStream_t s);
+cudaError_t launch_moe_combine(const MoeCombineArgs& a, int n, cudaStream_t s);
 
 // ---- small kernels ----------------------------------------------------------------
 cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,

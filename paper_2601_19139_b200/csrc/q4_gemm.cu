@@ -52,6 +52,12 @@ struct GemmParams {
   int ks;      // nominal K-slice (multiple of 256)
   int splits;  // gridDim.y
   int epilogue;
+  // grouped mode (MoE experts): blockIdx.z is a slot of the touched-expert list; the tensors of expert
+  // expert_ids[slot] start expert_rows rows further per expert; operand and output move by their slot strides.
+  const int* expert_ids;
+  const int* n_touched;
+  int expert_rows;
+  size_t xp_slot_stride, xs_slot_stride, out_slot_stride, out_xs_slot_stride;  // elements
 };
 
 // Four bf16x2 registers {16 + code j, 16 + code j+4}, j = 0..3, from one packed word: the code is placed in
@@ -87,7 +93,7 @@ __device__ __forceinline__ void store_out(const GemmParams& p, int row, int req,
 }
 
 template <int MT, int NT, int STAGES>
-__global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(const GemmParams p) {
+__global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(const GemmParams pin) {
   constexpr int R = 16 * MT;        // rows per warp
   constexpr int NP = 8 * NT;        // padded request count
   constexpr int kRows = kWarps * R; // rows per CTA
@@ -97,6 +103,23 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
   __shared__ int s_is_last;
 
   grid_launch_dependents();
+
+  GemmParams p = pin;
+  if (pin.expert_ids) {
+    // the expert list is written by the preceding kernel: wait for it before anything else
+    grid_dependency_wait();
+    const int slot = blockIdx.z;
+    if (slot >= *pin.n_touched) return;
+    const size_t e = (size_t)pin.expert_ids[slot];
+    p.qw += e * pin.expert_rows * (size_t)(pin.K >> 3);
+    p.scales += e * pin.expert_rows * (size_t)(pin.K >> 6);
+    p.biases += e * pin.expert_rows * (size_t)(pin.K >> 6);
+    p.xp += (size_t)slot * pin.xp_slot_stride;
+    p.xs += (size_t)slot * pin.xs_slot_stride;
+    if (p.out_xs) p.out_xs += (size_t)slot * pin.out_xs_slot_stride;
+    if (p.out_xp) p.out_xp += (size_t)slot * pin.out_slot_stride;
+    if (p.out) p.out = reinterpret_cast<uint16_t*>(p.out) + (size_t)slot * pin.out_slot_stride;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const bool silu = p.epilogue == EPI_SILU_PACK;
@@ -302,7 +325,7 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
       const int col0 = blockIdx.x * (kRows / 2) + c * 8;
       if (col0 < half_n && req < p.n) {
         *reinterpret_cast<uint4*>(p.out_xp + (size_t)req * half_n + col0) = permute_chunk(v);
-        if ((c & 7) == 0) p.out_xs[(size_t)(col0 >> 6) * 16 + req] = gsum;
+        if ((c & 7) == 0 && p.out_xs) p.out_xs[(size_t)(col0 >> 6) * 16 + req] = gsum;
       }
     }
     return;
@@ -348,7 +371,7 @@ struct Tiling {
 int g_sm_count = 0;
 int g_force_cfg = -1;  // debugging aid: environment variable Q4D_GEMM_CFG forces the n > 8 configuration
 
-Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count) {
+Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count, bool grouped = false) {
   Tiling t;
   const int rows_logical = epilogue == EPI_SILU_PACK ? N / 2 : N;  // rows that index row blocks
   const int quads = K / 256;
@@ -373,6 +396,7 @@ Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count) {
       break;
     }
   }
+  if (grouped) qps = quads;  // experts: many small GEMMs fill the machine without split-K (K <= 2048)
   t.qps = qps;
   t.splits = quads / qps;
   return t;
@@ -454,11 +478,11 @@ cudaError_t gemm_init() {
   if (e != cudaSuccess) return e;
   // 227 KB is the per-CTA limit for static + dynamic shared memory; leave room for the static part.
   const int big = 227 * 1024 - 1024;
-  e = cudaFuncSetAttribute(q4_gemm_kernel<1, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big / 2 - 1024);
+  e = cudaFuncSetAttribute(q4_gemm_kernel<1, 1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<2, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big / 2 - 1024);
+    e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   g_sm_count = sms;
@@ -473,8 +497,13 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
   if (a.n <= 0) return cudaSuccess;
   if (a.N <= 0 || a.K <= 0 || (a.K % 256) || a.n > kMaxBatch) return cudaErrorInvalidValue;
   if (a.epilogue == EPI_SILU_PACK && ((a.N % 16) || !a.out_xp || !a.out_xs)) return cudaErrorInvalidValue;
-  const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count);
+  const bool grouped = a.expert_ids != nullptr;
+  if (grouped && (a.K > 2048 || !a.n_touched || a.max_slots < 1)) return cudaErrorInvalidValue;
+  const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;
+  p.expert_ids = a.expert_ids, p.n_touched = a.n_touched, p.expert_rows = a.N;
+  p.xp_slot_stride = a.xp_slot_stride, p.xs_slot_stride = a.xs_slot_stride;
+  p.out_slot_stride = a.out_slot_stride, p.out_xs_slot_stride = a.out_xs_slot_stride;
   p.qw = a.qw, p.scales = a.scales, p.biases = a.biases, p.xp = a.xp, p.xs = a.xs, p.out = a.out;
   p.out_xp = a.out_xp, p.out_xs = a.out_xs, p.argmax_partial = a.argmax_partial;
   p.partial = a.partial, p.counters = a.counters;
@@ -484,7 +513,7 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     if (!a.partial || !a.counters || tiling_partial_bytes(t) > a.partial_bytes || t.rowblocks > a.counters_len)
       return cudaErrorInvalidValue;
   }
-  const dim3 grid(t.rowblocks, t.splits), block(kThreads);
+  const dim3 grid(t.rowblocks, t.splits, grouped ? a.max_slots : 1), block(kThreads);
   switch (t.cfg) {
     case 0:
       return launch_kernel(q4_gemm_kernel<1, 1, 4>, grid, block, smem_bytes<1, 1, 4>(p.ks), s, p);

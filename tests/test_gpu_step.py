@@ -65,6 +65,7 @@ def _run_steps(q4d, sc, steps):
     logits = torch.zeros(n, shape.vocab, dtype=torch.float32, device="cuda")
     agree = total = 0
     worst_max = worst_rms = 0.0
+    sc.per_request_max = []
     toks = sc.tokens.copy()
     for _ in range(steps):
         bt = sc.block_tables()
@@ -73,6 +74,7 @@ def _run_steps(q4d, sc, steps):
         o_next, o_logits, _ = sc.oracle.decode_step(sc.host_pool, 16, sc.lens, toks, bt)
         emax, erms = _logit_err(logits.cpu().numpy(), o_logits)
         worst_max, worst_rms = max(worst_max, float(emax.max())), max(worst_rms, float(erms.max()))
+        sc.per_request_max.extend(float(v) for v in emax)
         agree += int((nxt.cpu().numpy() == o_next).sum())
         total += n
         for r in range(n):
@@ -148,16 +150,37 @@ TOYS = [
 ]
 
 
-@pytest.mark.parametrize("shape,lens", TOYS, ids=[t[0].name for t in TOYS])
+# Mixture-of-experts layers (router, top-k, routed experts, weighted combination)
+MOE_TOYS = [
+    (shapes.toy("gpu-toy-moe-small", hidden=256, n_q_heads=4, n_kv_heads=2, mlp_inter=256, vocab=1024, n_experts=8,
+                top_k=2, expert_inter=256, norm_topk_prob=1), [0, 15, 16, 40, 7]),
+    (shapes.toy("gpu-toy-moe-wide", hidden=512, n_q_heads=8, n_kv_heads=2, mlp_inter=256, vocab=2000, n_experts=40,
+                top_k=8, expert_inter=768, norm_topk_prob=0),
+     [3, 100, 31, 64, 9, 200, 1, 0, 22, 50, 12, 47, 8, 63, 15, 16]),
+    (shapes.toy("gpu-toy-moe-1req", n_layers=1, hidden=2048, n_q_heads=4, n_kv_heads=1, mlp_inter=256, vocab=1024,
+                n_experts=128, top_k=8, expert_inter=768, norm_topk_prob=1), [33]),
+]
+
+
+@pytest.mark.parametrize("shape,lens", TOYS + MOE_TOYS, ids=[t[0].name for t in TOYS + MOE_TOYS])
 def test_toy_whole_steps_match_oracle(q4d, shape, lens):
     """Shallow models: the whole step, free-running.  Up to two layers the logit tolerance is met directly; beyond
     that the drift bound applies."""
     sc = Scenario(shape, lens, seed=3)
     agree, total, worst_max, worst_rms = _run_steps(q4d, sc, steps=4)
     rms_b, max_b = drift_bounds(shape.n_layers)
+    assert agree >= total - max(1, total // 50), (agree, total)
+    if shape.n_experts:
+        # Top-k routing is a discontinuous decision: where the k-th and (k+1)-th router logits of a request are
+        # closer than the rounding noise of the layers before, the two sides may pick different experts and that
+        # request's logits move by several per cent (the oracle does the same against itself when only its
+        # accumulation precision changes).  So: nearly all requests within the tolerance, the few others bounded.
+        e = np.array(sc.per_request_max)
+        assert (e <= LOGIT_TOL).mean() >= 0.9, np.sort(e)[-8:]
+        assert worst_max <= 0.15, worst_max
+        return
     assert worst_max <= (LOGIT_TOL if shape.n_layers <= 2 else max_b), worst_max
     assert worst_rms <= rms_b, worst_rms
-    assert agree >= total - max(1, total // 50), (agree, total)
 
 
 @pytest.mark.parametrize("production", [True, False], ids=["step-path", "composed-ops"])
@@ -165,6 +188,15 @@ def test_toy_whole_steps_match_oracle(q4d, shape, lens):
 def test_toy_layers_match_oracle_teacher_forced(q4d, shape, lens, production):
     sc = Scenario(shape, lens, seed=4)
     _, emax, same, n = _layerwise(q4d, sc, production)
+    assert emax <= LOGIT_TOL and same == n
+
+
+@pytest.mark.parametrize("shape,lens", MOE_TOYS, ids=[t[0].name for t in MOE_TOYS])
+def test_moe_layers_match_oracle_teacher_forced(q4d, shape, lens):
+    """The routed-expert layers through the step's own launch sequence, each from the oracle's input: a wrong
+    expert, weight or slot would move whole rows far outside the rounding band."""
+    sc = Scenario(shape, lens, seed=5)
+    _, emax, same, n = _layerwise(q4d, sc, production=True)
     assert emax <= LOGIT_TOL and same == n
 
 
@@ -182,6 +214,18 @@ def test_qwen3_0p6b_layers_and_head_teacher_forced(q4d):
         del sc
         torch.cuda.empty_cache()
     assert agree / total >= 0.995, (agree, total)
+
+
+def test_moe_30b_shape_layers_and_head_teacher_forced(q4d):
+    """The MoE-30B layer at full width (128 experts, 8 per token, 768-wide experts, hidden 2048) and the full
+    vocabulary head, two layers deep, 16 requests: each layer from the oracle's input."""
+    import dataclasses
+    shape = dataclasses.replace(shapes.MOE_30B, name="moe-30b-a3b-shaped-2layers", n_layers=2)
+    rng = np.random.default_rng(1)
+    lens = gen.draw_lengths(16, 128, 2048, rng).tolist()
+    sc = Scenario(shape, lens, seed=6)
+    _, emax, same, n = _layerwise(q4d, sc)
+    assert emax <= LOGIT_TOL and same == n
 
 
 def test_qwen3_0p6b_single_request_step(q4d):
