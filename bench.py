@@ -6,7 +6,8 @@ leaving and four joining (512 prefilled tokens) every 32 steps; `--workload` sel
 
   value      tokens/s with everything resident in HBM (tokens chained on the device, no host sync)
   e2e        tokens/s through q4d_decode_step_host: host inputs, host outputs, a sync per step
-  roofline   the dominant kernel (paged attention) timed with CUDA events around each of its launches
+  roofline   the dominant kernel (the persistent whole-step kernel of dense models) timed with CUDA events
+             around each of its launches
   cpu_baseline  the CPU oracle on a bounded sample of the same step, on the host cores
 
 `--impl reference` times the CPU oracle alone (the only reference implementation there is).
@@ -284,25 +285,42 @@ def main():
     barrier()
     h2d, d2h = model.step_io_bytes()
 
-    # ---- per-kernel timing (events around every launch) for the roofline of the dominant kernel ----
+    # ---- per-launch timing (events around every launch) for the roofline of the dominant kernel ----
+    fused = model.is_fused()
     model.profile_enable(True)
+    if fused:
+        model.timeline_enable(True)
     bytes_log.clear()
     for _ in range(args.profile_steps):
         one_step("chained")
     torch.cuda.synchronize()
     prof = model.profile_read()
     model.profile_enable(False)
-    kv_read_layer = float(np.mean([b["kv_read"] for b in bytes_log])) / shape.n_layers
-    att_ms, att_cnt = prof["attention"]
     peak, peak_kind = peaks()
-    total_prof_ms = sum(v[0] for v in prof.values())
-    kernels = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
-                   "share": v[0] / total_prof_ms} for k, v in prof.items() if v[1]}
-    att_gbs = kv_read_layer / (att_ms / att_cnt * 1e-3) / 1e9 if att_cnt else 0.0
-    roofline = {"kernel": "paged_attention_kernel", "bound": "hbm", "achieved": att_gbs, "peak": peak, "unit": "GB/s",
-                "frac": att_gbs / peak, "peak_kind": peak_kind, "traffic": None,
-                "bytes_per_launch": kv_read_layer, "us_per_launch": att_ms / max(att_cnt, 1) * 1e3,
-                "timing": "CUDA events around each launch, profile pass right after the timed steps"}
+    if fused:
+        # one persistent kernel runs the whole step: its algorithmic bytes are the step's
+        step_ms, step_cnt = prof["fused_step"]
+        per_launch = float(np.mean([b["total"] for b in bytes_log]))
+        gbs = per_launch / (step_ms / step_cnt * 1e-3) / 1e9 if step_cnt else 0.0
+        roofline = {"kernel": "fused_step_kernel", "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s",
+                    "frac": gbs / peak, "peak_kind": peak_kind, "traffic": None, "bytes_per_launch": per_launch,
+                    "us_per_launch": step_ms / max(step_cnt, 1) * 1e3,
+                    "timing": "CUDA events around each launch, profile pass right after the timed steps"}
+        tl = model.timeline_read()      # phases of the last profiled step, from the kernel's own clock stamps
+        model.timeline_enable(False)
+        tl_total = sum(v[0] for v in tl.values()) or 1.0
+        kernels = {k: {"us_per_step": v[0], "phases_per_step": v[1], "share": v[0] / tl_total} for k, v in tl.items()}
+    else:
+        kv_read_layer = float(np.mean([b["kv_read"] for b in bytes_log])) / shape.n_layers
+        att_ms, att_cnt = prof["attention"]
+        total_prof_ms = sum(v[0] for v in prof.values())
+        kernels = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
+                       "share": v[0] / total_prof_ms} for k, v in prof.items() if v[1]}
+        att_gbs = kv_read_layer / (att_ms / att_cnt * 1e-3) / 1e9 if att_cnt else 0.0
+        roofline = {"kernel": "paged_attention_kernel", "bound": "hbm", "achieved": att_gbs, "peak": peak,
+                    "unit": "GB/s", "frac": att_gbs / peak, "peak_kind": peak_kind, "traffic": None,
+                    "bytes_per_launch": kv_read_layer, "us_per_launch": att_ms / max(att_cnt, 1) * 1e3,
+                    "timing": "CUDA events around each launch, profile pass right after the timed steps"}
 
     # ---- max over ranks, aggregate ----
     if dist is not None:

@@ -192,7 +192,7 @@ int q4d_decode_step_host(q4d_model* model, q4d_kv_pool* pool, int32_t n, const i
 enum {
   Q4D_K_EMBED = 0, Q4D_K_RMSNORM, Q4D_K_GEMM_QKV, Q4D_K_ROPE_APPEND, Q4D_K_ATTENTION,
   Q4D_K_ATTN_MERGE, Q4D_K_GEMM_O, Q4D_K_GEMM_GATE_UP, Q4D_K_GEMM_DOWN, Q4D_K_MOE_ROUTER,
-  Q4D_K_MOE_GATE_UP, Q4D_K_MOE_DOWN, Q4D_K_LM_HEAD, Q4D_K_ARGMAX, Q4D_K_COUNT
+  Q4D_K_MOE_GATE_UP, Q4D_K_MOE_DOWN, Q4D_K_LM_HEAD, Q4D_K_ARGMAX, Q4D_K_FUSED_STEP, Q4D_K_COUNT
 };
 /* With profiling on, every kernel launch of a step is bracketed by CUDA events
  * on the step's stream.  q4d_profile_read synchronises, adds up the elapsed
@@ -202,6 +202,18 @@ int q4d_profile_enable(q4d_model* model, int32_t on);
 int q4d_profile_read(q4d_model* model, float* ms, int32_t* launches);
 /* Kernel launches enqueued by this model since creation. */
 int64_t q4d_launch_count(q4d_model* model);
+/* 1 if the model runs a step as one persistent kernel (dense models; every phase of the step in one
+ * cooperative launch, class Q4D_K_FUSED_STEP in the profile), 0 if it launches one kernel per operation
+ * (mixture-of-experts models, or the environment variable Q4D_UNFUSED=1 at model creation). */
+int q4d_step_is_fused(q4d_model* model);
+/* Phase timeline of the persistent kernel.  While enabled, the kernel stamps the nanosecond clock after
+ * every grid barrier.  q4d_timeline_read synchronises the device and adds up, for the most recent step,
+ * the microseconds and the number of phases per class into us[Q4D_K_COUNT], phases[Q4D_K_COUNT] (host
+ * arrays); a phase is filed under the class of the kernel it replaces (attention includes qk-norm, rotary
+ * embedding, append and merge; projections include the RMSNorm they read through; the LM head includes the
+ * argmax).  All zeros for a model that is not fused. */
+int q4d_timeline_enable(q4d_model* model, int32_t on);
+int q4d_timeline_read(q4d_model* model, float* us, int32_t* phases);
 /* Bytes the most recent step copied host -> device (per-step metadata: tokens,
  * lengths, block tables, attention work list) and device -> host (only the
  * host-output variant copies anything back). */

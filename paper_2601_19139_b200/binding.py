@@ -15,13 +15,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libq4decode.so")
 
 K_NAMES = ["embed", "rmsnorm", "gemm_qkv", "rope_append", "attention", "attn_merge", "gemm_o", "gemm_gate_up",
-           "gemm_down", "moe_router", "moe_gate_up", "moe_down", "lm_head", "argmax"]
+           "gemm_down", "moe_router", "moe_gate_up", "moe_down", "lm_head", "argmax", "fused_step"]
 
 EXPORTS = [
     "q4d_last_error", "q4d_model_workspace_bytes", "q4d_model_create", "q4d_model_destroy", "q4d_kv_pool_bytes",
     "q4d_kv_pool_create", "q4d_kv_pool_destroy", "q4d_request_admit", "q4d_request_release", "q4d_request_len",
     "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_profile_enable",
-    "q4d_profile_read", "q4d_launch_count", "q4d_step_io_bytes", "q4d_op_scratch_bytes", "q4d_q4_gemm",
+    "q4d_profile_read", "q4d_launch_count", "q4d_step_is_fused", "q4d_timeline_enable", "q4d_timeline_read",
+    "q4d_step_io_bytes", "q4d_op_scratch_bytes", "q4d_q4_gemm",
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
     "q4d_rmsnorm", "q4d_embed", "q4d_rope_append", "q4d_paged_attention", "q4d_argmax", "q4d_debug_dequant",
     "q4d_debug_kv_gather", "q4d_debug_run_layers",
@@ -160,6 +161,18 @@ class Model:
 
     def launch_count(self):
         return int(lib().q4d_launch_count(self.handle))
+
+    def is_fused(self):
+        return bool(lib().q4d_step_is_fused(self.handle))
+
+    def timeline_enable(self, on=True):
+        _check(lib().q4d_timeline_enable(self.handle, int(on)))
+
+    def timeline_read(self):
+        us = (C.c_float * len(K_NAMES))()
+        cnt = (C.c_int32 * len(K_NAMES))()
+        _check(lib().q4d_timeline_read(self.handle, us, cnt))
+        return {k: (float(us[i]), int(cnt[i])) for i, k in enumerate(K_NAMES) if cnt[i]}
 
     def step_io_bytes(self):
         h2d, d2h = C.c_int64(), C.c_int64()

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "../../include/q4decode.h"
+#include "fused_step.h"
 #include "kernels.h"
 
 using namespace q4d;
@@ -66,7 +67,32 @@ struct Workspace {
   // MoE: plain normed state, routing results, touched-expert list, per-slot expert activations and outputs
   size_t yplain, m_idx, m_wgt, m_ints, m_hp, m_hs, m_o;
   int counters_len, amax_blocks;
+  // persistent whole-step kernel (dense models): plain attention output and gated MLP activations, sums of squares
+  // of the residual stream, split-KV scratch, argmax partials, barrier/status words, phase table
+  size_t f_attn, f_h, f_ss, f_pacc, f_pml, f_attn_counters, f_amax, f_control, f_phases, f_timeline;
+  int f_max_items, f_max_ctas, f_n_phases;
 };
+
+// The CTA count the whole-step kernel is sized for: one per SM of the current device (148 when there is none).
+int fused_cta_bound() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  return sms > 0 ? sms : 148;
+}
+
+struct FusedGemmDims {
+  int N, K, ntiles, S;
+};
+FusedGemmDims fused_dims(int N, int K, int epi) {
+  FusedGemmDims d;
+  d.N = N, d.K = K;
+  d.ntiles = epi == EPI_SILU_PACK ? N / 16 : (N + 15) / 16;  // SiLU tiles: 8 gate rows + 8 up rows of N/2 columns
+  d.S = (K + kFusedSliceK - 1) / kFusedSliceK;
+  return d;
+}
 
 bool shape_supported(const q4d_shape& s, std::string* why) {
   auto bad = [&](const char* m) {
@@ -146,6 +172,25 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   w.part_acc = take((size_t)ml.max_work * s.n_q_heads * kHeadDim * 4);
   w.part_ml = take((size_t)ml.max_work * s.n_q_heads * 2 * 4);
   w.meta = take(ml.bytes);
+  w.f_attn = w.f_h = w.f_ss = w.f_pacc = w.f_pml = w.f_attn_counters = w.f_amax = 0;
+  w.f_control = w.f_phases = w.f_timeline = 0;
+  w.f_max_items = w.f_max_ctas = w.f_n_phases = 0;
+  if (!s.n_experts) {
+    const int G = s.n_q_heads / s.n_kv_heads;
+    w.f_max_ctas = fused_cta_bound();
+    w.f_max_items = std::max(w.f_max_ctas * 8, 16 * s.n_kv_heads);
+    w.f_n_phases = 3 + kFusedPhasesPerLayer * s.n_layers;
+    w.f_attn = take(B * qdim * 2);
+    w.f_h = take(B * (size_t)s.mlp_inter * 2);
+    w.f_ss = take((size_t)(s.hidden / 16) * 16 * 4);
+    w.f_pacc = take((size_t)w.f_max_items * G * kHeadDim * 4);
+    w.f_pml = take((size_t)w.f_max_items * G * 2 * 4);
+    w.f_attn_counters = take((size_t)16 * s.n_kv_heads * 4);
+    w.f_amax = take((size_t)w.f_max_ctas * 16 * sizeof(float2));
+    w.f_control = take(256);
+    w.f_phases = take((size_t)w.f_n_phases * sizeof(FusedPhase));
+    w.f_timeline = take((size_t)(w.f_n_phases + 1) * 8);
+  }
   w.bytes = o;
   return w;
 }
@@ -179,6 +224,14 @@ struct q4d_model {
   int64_t launches;
   int64_t last_h2d, last_d2h;
   int32_t* host_next;  // pinned, for the host-output variant
+  // persistent whole-step kernel
+  bool fused;
+  int fused_ctas;
+  FusedDims fused_dims[kFusedDimKinds];
+  bool timeline;
+  uint32_t* host_status;  // pinned copy of the kernel's status word, read back after every step
+  cudaEvent_t status_done;
+  bool status_pending;
 };
 
 struct q4d_kv_pool {
@@ -234,6 +287,137 @@ GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint1
 
 bool qt_ok(const q4d_qtensor& t) { return t.q && t.scales && t.biases; }
 
+// ---- persistent whole-step kernel: phase table and per-step launch ----
+
+void build_fused_phases(const q4d_model* m, std::vector<FusedPhase>* out) {
+  const q4d_shape& sh = m->sh;
+  const int H = sh.hidden, nq = sh.n_q_heads, nkv = sh.n_kv_heads, I = sh.mlp_inter, V = sh.vocab;
+  const int nqkv = (nq + 2 * nkv) * kHeadDim, qdim = nq * kHeadDim;
+  uint16_t* x = reinterpret_cast<uint16_t*>(m->ws + m->lay.x);
+  uint16_t* qkv = reinterpret_cast<uint16_t*>(m->ws + m->lay.qkv);
+  uint16_t* attn = reinterpret_cast<uint16_t*>(m->ws + m->lay.f_attn);
+  uint16_t* h = reinterpret_cast<uint16_t*>(m->ws + m->lay.f_h);
+  uint16_t* y = reinterpret_cast<uint16_t*>(m->ws + m->lay.yp);  // normed hidden state, fragment order
+  auto gemm = [&](const q4d_qtensor& t, int N, int K, int epi, const uint16_t* in, void* o, int out_stride, int cls) {
+    FusedPhase P = {};
+    const FusedGemmDims d = fused_dims(N, K, epi);
+    P.type = PH_GEMM, P.epi = epi, P.N = N, P.K = K, P.ntiles = d.ntiles, P.S = d.S;
+    P.qw = t.q, P.scales = t.scales, P.biases = t.biases;
+    P.in = in, P.out = o, P.out_stride = out_stride, P.cls = cls;
+    out->push_back(P);
+  };
+  auto norm = [&](const uint16_t* w, int cls) {
+    FusedPhase P = {};
+    P.type = PH_NORM, P.K = H, P.in = x, P.norm_w = w, P.out = y, P.cls = cls;
+    out->push_back(P);
+  };
+  out->clear();
+  FusedPhase E = {};
+  E.type = PH_EMBED, E.cls = Q4D_K_EMBED;
+  out->push_back(E);
+  for (int l = 0; l < sh.n_layers; ++l) {
+    const q4d_layer_weights& lw = m->layers[l];
+    norm(lw.attn_norm, Q4D_K_RMSNORM);
+    gemm(lw.wqkv, nqkv, H, EPI_BF16, y, qkv, nqkv, Q4D_K_GEMM_QKV);
+    FusedPhase A = {};
+    A.type = PH_ATTN, A.layer = l, A.cls = Q4D_K_ATTENTION;
+    A.q_norm = sh.qk_norm ? lw.q_norm : nullptr, A.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
+    out->push_back(A);
+    gemm(lw.wo, H, qdim, EPI_RESIDUAL, attn, x, H, Q4D_K_GEMM_O);
+    norm(lw.mlp_norm, Q4D_K_RMSNORM);
+    gemm(lw.w_gate_up, 2 * I, H, EPI_SILU_PACK, y, h, I, Q4D_K_GEMM_GATE_UP);
+    gemm(lw.w_down, H, I, EPI_RESIDUAL, h, x, H, Q4D_K_GEMM_DOWN);
+  }
+  norm(m->w.final_norm, Q4D_K_RMSNORM);
+  gemm(m->w.lm_head, V, H, EPI_F32, y, nullptr, V, Q4D_K_LM_HEAD);
+}
+
+// Reports a barrier timeout of an earlier step once its status word has come back.
+int fused_check_status(q4d_model* m, bool wait) {
+  if (!m->status_pending) return Q4D_OK;
+  cudaError_t e = wait ? cudaEventSynchronize(m->status_done) : cudaEventQuery(m->status_done);
+  if (e == cudaErrorNotReady) return Q4D_OK;
+  if (e != cudaSuccess) return fail_cuda(e, "status read-back");
+  m->status_pending = false;
+  if (*m->host_status != 0u)
+    return fail(Q4D_ERR_TIMEOUT, "decode_step: a grid barrier of an earlier step timed out; destroy and re-create the model");
+  return Q4D_OK;
+}
+
+int run_fused(q4d_model* m, q4d_kv_pool* pool, int n, const int32_t* lens, const int32_t* d_tokens, const int32_t* d_bt,
+              int32_t* next_dev, float* logits_dev, cudaStream_t s, int layer_begin, int layer_end, const uint16_t* x_in,
+              uint16_t* x_out, bool ranged) {
+  const q4d_shape& sh = m->sh;
+  const Workspace& lay = m->lay;
+  FusedStep fp = {};
+  fp.phases = at<FusedPhase>(m, lay.f_phases);
+  fp.n = n, fp.tokens = d_tokens, fp.bt = d_bt, fp.max_blocks = m->ml.max_blocks_cap;
+  fp.n_phases = lay.f_n_phases;
+  for (int i = 0; i < kFusedDimKinds; ++i) fp.dims[i] = m->fused_dims[i];
+  // attention plan: equal chunks of whole blocks, at most one (request, chunk, kv head) item per warp of the grid
+  const int W = m->fused_ctas * 8, nkv = sh.n_kv_heads;
+  long long total = 0;
+  int nb[kMaxBatch], maxnb = 1;
+  for (int r = 0; r < n; ++r) {
+    fp.lens[r] = lens[r];
+    nb[r] = (lens[r] + 1 + kBlockSize - 1) / kBlockSize;
+    total += nb[r];
+    maxnb = std::max(maxnb, nb[r]);
+  }
+  int C = (int)std::max<long long>(1, (total * nkv + W - 1) / W);
+  for (;; ++C) {
+    long long items = 0;
+    for (int r = 0; r < n; ++r) items += (long long)((nb[r] + C - 1) / C) * nkv;
+    if (items <= W || C >= maxnb) break;
+  }
+  fp.chunk_blocks = C;
+  fp.item_prefix[0] = 0;
+  for (int r = 0; r < n; ++r) fp.item_prefix[r + 1] = fp.item_prefix[r] + ((nb[r] + C - 1) / C) * nkv;
+  for (int r = n; r < kMaxBatch; ++r) fp.item_prefix[r + 1] = fp.item_prefix[n];
+  fp.n_items = fp.item_prefix[n];
+  if (fp.n_items > lay.f_max_items) return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "decode_step: split-KV scratch too small");
+  fp.H = sh.hidden, fp.nq = sh.n_q_heads, fp.nkv = nkv, fp.V = sh.vocab, fp.eps = sh.rms_eps;
+  fp.rope = m->w.rope_cos_sin;
+  fp.embed_q = m->w.embed.q, fp.embed_s = m->w.embed.scales, fp.embed_b = m->w.embed.biases;
+  fp.pool = pool->mem;
+  fp.layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
+  fp.x = at<uint16_t>(m, lay.x), fp.qkv = at<uint16_t>(m, lay.qkv), fp.attn = at<uint16_t>(m, lay.f_attn);
+  fp.ss = at<float>(m, lay.f_ss);
+  fp.pacc = at<float>(m, lay.f_pacc), fp.pml = at<float>(m, lay.f_pml);
+  fp.attn_counters = at<int>(m, lay.f_attn_counters), fp.amax = at<float2>(m, lay.f_amax);
+  fp.next = next_dev, fp.logits = logits_dev;
+  fp.control = at<unsigned int>(m, lay.f_control);
+  fp.timeline = m->timeline ? at<unsigned long long>(m, lay.f_timeline) : nullptr;
+
+  auto launch = [&](int ph_begin, int ph_end, int from_x) -> int {
+    fp.ph_begin = ph_begin, fp.ph_end = ph_end, fp.embed_from_x = from_x;
+    cudaError_t e = cudaMemsetAsync(fp.control, 0, sizeof(unsigned int), s);  // barrier arrivals; the status word stays
+    if (e != cudaSuccess) return fail_cuda(e, "barrier reset");
+    e = timed(m, Q4D_K_FUSED_STEP, s, [&]() -> cudaError_t { return launch_fused_step(fp, m->fused_ctas, s); });
+    return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "fused step launch");
+  };
+  int rc = Q4D_OK;
+  if (!ranged) {
+    rc = launch(0, lay.f_n_phases, 0);
+  } else {
+    cudaError_t ce = cudaMemcpyAsync(fp.x, x_in, (size_t)n * sh.hidden * 2, cudaMemcpyDeviceToDevice, s);
+    if (ce != cudaSuccess) return fail_cuda(ce, "hidden state copy");
+    rc = launch(0, 1, 1);  // sums of squares of the given hidden state
+    if (rc == Q4D_OK && layer_end > layer_begin) rc = launch(1 + kFusedPhasesPerLayer * layer_begin, 1 + kFusedPhasesPerLayer * layer_end, 0);
+    if (rc != Q4D_OK) return rc;
+    ce = cudaMemcpyAsync(x_out, fp.x, (size_t)n * sh.hidden * 2, cudaMemcpyDeviceToDevice, s);
+    if (ce != cudaSuccess) return fail_cuda(ce, "hidden state copy");
+  }
+  if (rc != Q4D_OK) return rc;
+  if (!m->status_pending) {
+    cudaError_t e = cudaMemcpyAsync(m->host_status, fp.control + 1, sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaEventRecord(m->status_done, s);
+    if (e != cudaSuccess) return fail_cuda(e, "status read-back");
+    m->status_pending = true;
+  }
+  return Q4D_OK;
+}
+
 // The launch sequence of a step.  A whole step embeds the tokens, runs every layer and the head, and advances the
 // requests.  The parity export runs only layers [layer_begin, layer_end) from a given hidden state (x_in) and
 // returns the hidden state (x_out) without advancing anything.
@@ -254,6 +438,10 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   if (!ids || !bt || max_blocks < 1 || (!range && ((!tokens_host && !tokens_dev) || !next_dev)))
     return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL argument");
   const q4d_shape& sh = m->sh;
+  if (m->fused) {
+    const int rc = fused_check_status(m, false);
+    if (rc != Q4D_OK) return rc;
+  }
 
   // ---- validate on the host; nothing is changed before this block passes ----
   int32_t lens[kMaxBatch];
@@ -305,7 +493,8 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     for (int i = 0; i < ml.max_blocks_cap; ++i)
       h_bt[(size_t)r * ml.max_blocks_cap + i] = i < need ? bt[(size_t)r * max_blocks + i] : 0;
   }
-  const AttnPlan plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
+  AttnPlan plan = {0, 0, 0};  // the whole-step kernel plans its attention items from the lengths alone
+  if (!m->fused) plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
   unsigned char* dmeta = m->ws + m->lay.meta;
   const size_t head_bytes = ml.off_work + (size_t)plan.n_work * sizeof(int4);
   const size_t bt_bytes = (size_t)n * ml.max_blocks_cap * 4;
@@ -320,6 +509,15 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   const int32_t* d_tokens = tokens_dev ? tokens_dev : reinterpret_cast<const int32_t*>(dmeta + ml.off_tokens);
   const int32_t* d_lens = reinterpret_cast<const int32_t*>(dmeta + ml.off_lens);
   const int32_t* d_bt = reinterpret_cast<const int32_t*>(dmeta + ml.off_bt);
+
+  if (m->fused) {
+    const int rc = run_fused(m, pool, n, lens, d_tokens, d_bt, next_dev, logits_dev, s, range ? range->begin : 0,
+                             range ? range->end : 0, range ? range->x_in : nullptr, range ? range->x_out : nullptr,
+                             range != nullptr);
+    if (rc != Q4D_OK || range) return rc;
+    for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
+    return Q4D_OK;
+  }
 
   // ---- the launch sequence ----
   const int H = sh.hidden, nq = sh.n_q_heads, nkv = sh.n_kv_heads, I = sh.mlp_inter, V = sh.vocab;
@@ -490,6 +688,8 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   m->last_h2d = m->last_d2h = 0;
   m->staging_next = 0;
   m->host_next = nullptr;
+  m->fused = false, m->fused_ctas = 0, m->timeline = false;
+  m->host_status = nullptr, m->status_done = nullptr, m->status_pending = false;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -503,6 +703,30 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
   if (e == cudaSuccess && shape->n_experts)
     e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 2) * 4);
+  // Dense models run the whole step as one persistent kernel (Q4D_UNFUSED=1 selects the kernel-per-operation
+  // sequence instead; mixture-of-experts models always use it).
+  const char* unfused = getenv("Q4D_UNFUSED");
+  if (e == cudaSuccess && !shape->n_experts && !(unfused && unfused[0] == '1')) {
+    int max_ctas = 0;
+    e = fused_init(&max_ctas);
+    if (e == cudaSuccess && max_ctas > 0 && max_ctas <= lay.f_max_ctas) {
+      m->fused = true;
+      m->fused_ctas = max_ctas;
+      std::vector<FusedPhase> phases;
+      build_fused_phases(m, &phases);
+      for (int i = 0; i < kFusedDimKinds; ++i) {  // phase kinds: embedding, the phases of layer 0, final norm, LM head
+        const FusedPhase& P = phases[i < 8 ? i : phases.size() - 2 + (i - 8)];
+        FusedDims& D = m->fused_dims[i];
+        D.type = P.type, D.epi = P.epi, D.N = P.N, D.K = P.K, D.ntiles = P.ntiles, D.S = P.S, D.norm = P.norm, D.pad = 0;
+      }
+      e = cudaMemcpy(m->ws + lay.f_phases, phases.data(), phases.size() * sizeof(FusedPhase), cudaMemcpyHostToDevice);
+      if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_attn_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
+      if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_control, 0, 256);
+      if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->status_done, cudaEventDisableTiming);
+      if (e == cudaSuccess) *m->host_status = 0u;
+    }
+  }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     q4d_model_destroy(m);
@@ -519,6 +743,8 @@ int q4d_model_destroy(q4d_model* m) {
     if (m->staging_done[i]) cudaEventDestroy(m->staging_done[i]);
   }
   if (m->host_next) cudaFreeHost(m->host_next);
+  if (m->host_status) cudaFreeHost(m->host_status);
+  if (m->status_done) cudaEventDestroy(m->status_done);
   for (auto& r : m->prof_recs) cudaEventDestroy(r.a), cudaEventDestroy(r.b);
   for (auto ev : m->prof_free) cudaEventDestroy(ev);
   delete m;
@@ -607,7 +833,7 @@ int q4d_decode_step_host(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64
     return fail(Q4D_ERR_INVALID_ARG, "decode_step_host: NULL argument");
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int32_t* d_next = at<int32_t>(m, m->lay.next);
-  float* d_logits = at<float>(m, m->lay.logits);
+  float* d_logits = (logits_host || !m->fused) ? at<float>(m, m->lay.logits) : nullptr;
   const int rc = step_impl(m, pool, n, ids, last_tokens, nullptr, bt, max_blocks, d_next, d_logits, s);
   if (rc != Q4D_OK || n == 0) return rc;
   cudaError_t e = cudaMemcpyAsync(m->host_next, d_next, (size_t)n * 4, cudaMemcpyDeviceToHost, s);
@@ -615,6 +841,10 @@ int q4d_decode_step_host(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64
     e = cudaMemcpyAsync(logits_host, d_logits, (size_t)n * m->sh.vocab * 4, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail_cuda(e, "decode_step_host");
+  if (m->fused) {
+    const int st = fused_check_status(m, true);
+    if (st != Q4D_OK) return st;
+  }
   memcpy(next_tokens_host, m->host_next, (size_t)n * 4);
   m->last_d2h = (int64_t)n * 4 + (logits_host ? (int64_t)n * m->sh.vocab * 4 : 0);
   return Q4D_OK;
@@ -644,6 +874,35 @@ int q4d_profile_read(q4d_model* m, float* ms, int32_t* launches) {
 }
 
 int64_t q4d_launch_count(q4d_model* m) { return m ? m->launches : 0; }
+
+int q4d_step_is_fused(q4d_model* m) { return m && m->fused ? 1 : 0; }
+
+int q4d_timeline_enable(q4d_model* m, int32_t on) {
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "timeline_enable: NULL model");
+  m->timeline = on != 0 && m->fused;
+  return Q4D_OK;
+}
+
+int q4d_timeline_read(q4d_model* m, float* us, int32_t* phases) {
+  if (!m || !us || !phases) return fail(Q4D_ERR_INVALID_ARG, "timeline_read: NULL argument");
+  for (int i = 0; i < Q4D_K_COUNT; ++i) us[i] = 0.0f, phases[i] = 0;
+  if (!m->fused) return Q4D_OK;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return fail_cuda(e, "timeline_read");
+  const int np = m->lay.f_n_phases;
+  std::vector<unsigned long long> stamps(np + 1);
+  std::vector<FusedPhase> table(np);
+  e = cudaMemcpy(stamps.data(), m->ws + m->lay.f_timeline, stamps.size() * 8, cudaMemcpyDeviceToHost);
+  if (e == cudaSuccess) e = cudaMemcpy(table.data(), m->ws + m->lay.f_phases, table.size() * sizeof(FusedPhase), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(e, "timeline_read");
+  for (int i = 0; i < np; ++i) {
+    const int c = table[i].cls;
+    if (c < 0 || c >= Q4D_K_COUNT || stamps[i + 1] < stamps[i]) continue;
+    us[c] += (float)((double)(stamps[i + 1] - stamps[i]) * 1e-3);
+    phases[c] += 1;
+  }
+  return Q4D_OK;
+}
 
 int q4d_step_io_bytes(q4d_model* m, int64_t* h2d, int64_t* d2h) {
   if (!m || !h2d || !d2h) return fail(Q4D_ERR_INVALID_ARG, "step_io_bytes: NULL argument");
