@@ -69,7 +69,7 @@ struct Workspace {
   int counters_len, amax_blocks;
   // persistent whole-step kernel (dense models): plain attention output and gated MLP activations, sums of squares
   // of the residual stream, split-KV scratch, argmax partials, barrier/status words, phase table
-  size_t f_attn, f_h, f_ss, f_pacc, f_pml, f_attn_counters, f_amax, f_control, f_phases, f_timeline;
+  size_t f_attn, f_h, f_ss, f_pacc, f_pml, f_attn_counters, f_amax, f_control, f_timeline;
   int f_max_items, f_max_ctas, f_n_phases;
 };
 
@@ -173,22 +173,22 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   w.part_ml = take((size_t)ml.max_work * s.n_q_heads * 2 * 4);
   w.meta = take(ml.bytes);
   w.f_attn = w.f_h = w.f_ss = w.f_pacc = w.f_pml = w.f_attn_counters = w.f_amax = 0;
-  w.f_control = w.f_phases = w.f_timeline = 0;
+  w.f_control = w.f_timeline = 0;
   w.f_max_items = w.f_max_ctas = w.f_n_phases = 0;
   if (!s.n_experts) {
     const int G = s.n_q_heads / s.n_kv_heads;
     w.f_max_ctas = fused_cta_bound();
-    w.f_max_items = std::max(w.f_max_ctas * 8, 16 * s.n_kv_heads);
+    w.f_max_items = std::max(w.f_max_ctas * (kFusedThreads / 32), 16 * s.n_kv_heads);
     w.f_n_phases = 3 + kFusedPhasesPerLayer * s.n_layers;
     w.f_attn = take(B * qdim * 2);
     w.f_h = take(B * (size_t)s.mlp_inter * 2);
     w.f_ss = take((size_t)(s.hidden / 16) * 16 * 4);
-    w.f_pacc = take((size_t)w.f_max_items * G * kHeadDim * 4);
-    w.f_pml = take((size_t)w.f_max_items * G * 2 * 4);
+    const int Gs = (G + 1) & ~1;  // heads per split-KV partial result
+    w.f_pacc = take((size_t)w.f_max_items * Gs * kHeadDim * 4);
+    w.f_pml = take((size_t)w.f_max_items * Gs * 2 * 4);
     w.f_attn_counters = take((size_t)16 * s.n_kv_heads * 4);
     w.f_amax = take((size_t)w.f_max_ctas * 16 * sizeof(float2));
     w.f_control = take(256);
-    w.f_phases = take((size_t)w.f_n_phases * sizeof(FusedPhase));
     w.f_timeline = take((size_t)(w.f_n_phases + 1) * 8);
   }
   w.bytes = o;
@@ -227,7 +227,7 @@ struct q4d_model {
   // persistent whole-step kernel
   bool fused;
   int fused_ctas;
-  FusedDims fused_dims[kFusedDimKinds];
+  FusedStep* fused_params;  // host template of the kernel parameters
   bool timeline;
   uint32_t* host_status;  // pinned copy of the kernel's status word, read back after every step
   cudaEvent_t status_done;
@@ -289,47 +289,60 @@ bool qt_ok(const q4d_qtensor& t) { return t.q && t.scales && t.biases; }
 
 // ---- persistent whole-step kernel: phase table and per-step launch ----
 
-void build_fused_phases(const q4d_model* m, std::vector<FusedPhase>* out) {
+// Phase kinds of the whole-step kernel (index into FusedStep::dims) and the timeline class each is filed under.
+const int kFusedKindClass[kFusedDimKinds] = {Q4D_K_EMBED,  Q4D_K_RMSNORM,      Q4D_K_GEMM_QKV,  Q4D_K_ATTENTION, Q4D_K_GEMM_O,
+                                             Q4D_K_RMSNORM, Q4D_K_GEMM_GATE_UP, Q4D_K_GEMM_DOWN, Q4D_K_RMSNORM,   Q4D_K_LM_HEAD};
+int fused_kind(int ph, int n_phases) {
+  return ph == 0 ? 0 : (ph >= n_phases - 2 ? 8 + (ph - (n_phases - 2)) : 1 + (ph - 1) % kFusedPhasesPerLayer);
+}
+
+// Everything of the kernel's parameters that does not change from step to step.
+void build_fused_params(const q4d_model* m, FusedStep* fp) {
   const q4d_shape& sh = m->sh;
+  const Workspace& lay = m->lay;
   const int H = sh.hidden, nq = sh.n_q_heads, nkv = sh.n_kv_heads, I = sh.mlp_inter, V = sh.vocab;
   const int nqkv = (nq + 2 * nkv) * kHeadDim, qdim = nq * kHeadDim;
-  uint16_t* x = reinterpret_cast<uint16_t*>(m->ws + m->lay.x);
-  uint16_t* qkv = reinterpret_cast<uint16_t*>(m->ws + m->lay.qkv);
-  uint16_t* attn = reinterpret_cast<uint16_t*>(m->ws + m->lay.f_attn);
-  uint16_t* h = reinterpret_cast<uint16_t*>(m->ws + m->lay.f_h);
-  uint16_t* y = reinterpret_cast<uint16_t*>(m->ws + m->lay.yp);  // normed hidden state, fragment order
-  auto gemm = [&](const q4d_qtensor& t, int N, int K, int epi, const uint16_t* in, void* o, int out_stride, int cls) {
-    FusedPhase P = {};
-    const FusedGemmDims d = fused_dims(N, K, epi);
-    P.type = PH_GEMM, P.epi = epi, P.N = N, P.K = K, P.ntiles = d.ntiles, P.S = d.S;
-    P.qw = t.q, P.scales = t.scales, P.biases = t.biases;
-    P.in = in, P.out = o, P.out_stride = out_stride, P.cls = cls;
-    out->push_back(P);
-  };
-  auto norm = [&](const uint16_t* w, int cls) {
-    FusedPhase P = {};
-    P.type = PH_NORM, P.K = H, P.in = x, P.norm_w = w, P.out = y, P.cls = cls;
-    out->push_back(P);
-  };
-  out->clear();
-  FusedPhase E = {};
-  E.type = PH_EMBED, E.cls = Q4D_K_EMBED;
-  out->push_back(E);
+  memset(fp, 0, sizeof *fp);
   for (int l = 0; l < sh.n_layers; ++l) {
     const q4d_layer_weights& lw = m->layers[l];
-    norm(lw.attn_norm, Q4D_K_RMSNORM);
-    gemm(lw.wqkv, nqkv, H, EPI_BF16, y, qkv, nqkv, Q4D_K_GEMM_QKV);
-    FusedPhase A = {};
-    A.type = PH_ATTN, A.layer = l, A.cls = Q4D_K_ATTENTION;
-    A.q_norm = sh.qk_norm ? lw.q_norm : nullptr, A.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
-    out->push_back(A);
-    gemm(lw.wo, H, qdim, EPI_RESIDUAL, attn, x, H, Q4D_K_GEMM_O);
-    norm(lw.mlp_norm, Q4D_K_RMSNORM);
-    gemm(lw.w_gate_up, 2 * I, H, EPI_SILU_PACK, y, h, I, Q4D_K_GEMM_GATE_UP);
-    gemm(lw.w_down, H, I, EPI_RESIDUAL, h, x, H, Q4D_K_GEMM_DOWN);
+    FusedLayerPtrs& L = fp->layer[l];
+    const q4d_qtensor* t[4] = {&lw.wqkv, &lw.wo, &lw.w_gate_up, &lw.w_down};
+    for (int j = 0; j < 4; ++j) L.qw[j] = t[j]->q, L.scales[j] = t[j]->scales, L.biases[j] = t[j]->biases;
+    L.norm[0] = lw.attn_norm, L.norm[1] = lw.mlp_norm;
+    L.q_norm = sh.qk_norm ? lw.q_norm : nullptr, L.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
   }
-  norm(m->w.final_norm, Q4D_K_RMSNORM);
-  gemm(m->w.lm_head, V, H, EPI_F32, y, nullptr, V, Q4D_K_LM_HEAD);
+  fp->lm_qw = m->w.lm_head.q, fp->lm_scales = m->w.lm_head.scales, fp->lm_biases = m->w.lm_head.biases;
+  fp->final_norm = m->w.final_norm;
+  auto dims = [&](int kind, int type, int N, int K, int epi) {
+    FusedDims& D = fp->dims[kind];
+    D.type = type, D.epi = epi, D.N = N, D.K = K, D.norm = 0, D.pad = 0, D.ntiles = 0, D.S = 0;
+    if (type == PH_GEMM) {
+      const FusedGemmDims d = fused_dims(N, K, epi);
+      D.ntiles = d.ntiles, D.S = d.S;
+    }
+  };
+  dims(0, PH_EMBED, 0, H, 0);
+  dims(1, PH_NORM, 0, H, 0);
+  dims(2, PH_GEMM, nqkv, H, EPI_BF16);
+  dims(3, PH_ATTN, 0, 0, 0);
+  dims(4, PH_GEMM, H, qdim, EPI_RESIDUAL);
+  dims(5, PH_NORM, 0, H, 0);
+  dims(6, PH_GEMM, 2 * I, H, EPI_SILU_PACK);
+  dims(7, PH_GEMM, H, I, EPI_RESIDUAL);
+  dims(8, PH_NORM, 0, H, 0);
+  dims(9, PH_GEMM, V, H, EPI_F32);
+  fp->n_phases = lay.f_n_phases;
+  fp->H = H, fp->nq = nq, fp->nkv = nkv, fp->V = V, fp->eps = sh.rms_eps;
+  fp->rope = m->w.rope_cos_sin;
+  fp->embed_q = m->w.embed.q, fp->embed_s = m->w.embed.scales, fp->embed_b = m->w.embed.biases;
+  fp->x = reinterpret_cast<uint16_t*>(m->ws + lay.x), fp->y = reinterpret_cast<uint16_t*>(m->ws + lay.yp);
+  fp->h = reinterpret_cast<uint16_t*>(m->ws + lay.f_h), fp->qkv = reinterpret_cast<uint16_t*>(m->ws + lay.qkv);
+  fp->attn = reinterpret_cast<uint16_t*>(m->ws + lay.f_attn);
+  fp->ss = reinterpret_cast<float*>(m->ws + lay.f_ss);
+  fp->pacc = reinterpret_cast<float*>(m->ws + lay.f_pacc), fp->pml = reinterpret_cast<float*>(m->ws + lay.f_pml);
+  fp->attn_counters = reinterpret_cast<int*>(m->ws + lay.f_attn_counters);
+  fp->amax = reinterpret_cast<float2*>(m->ws + lay.f_amax);
+  fp->control = reinterpret_cast<unsigned int*>(m->ws + lay.f_control);
 }
 
 // Reports a barrier timeout of an earlier step once its status word has come back.
@@ -349,13 +362,10 @@ int run_fused(q4d_model* m, q4d_kv_pool* pool, int n, const int32_t* lens, const
               uint16_t* x_out, bool ranged) {
   const q4d_shape& sh = m->sh;
   const Workspace& lay = m->lay;
-  FusedStep fp = {};
-  fp.phases = at<FusedPhase>(m, lay.f_phases);
+  FusedStep& fp = *m->fused_params;  // the model's template; the per-step fields are filled in below
   fp.n = n, fp.tokens = d_tokens, fp.bt = d_bt, fp.max_blocks = m->ml.max_blocks_cap;
-  fp.n_phases = lay.f_n_phases;
-  for (int i = 0; i < kFusedDimKinds; ++i) fp.dims[i] = m->fused_dims[i];
   // attention plan: equal chunks of whole blocks, at most one (request, chunk, kv head) item per warp of the grid
-  const int W = m->fused_ctas * 8, nkv = sh.n_kv_heads;
+  const int W = m->fused_ctas * (kFusedThreads / 32), nkv = sh.n_kv_heads;
   long long total = 0;
   int nb[kMaxBatch], maxnb = 1;
   for (int r = 0; r < n; ++r) {
@@ -372,21 +382,16 @@ int run_fused(q4d_model* m, q4d_kv_pool* pool, int n, const int32_t* lens, const
   }
   fp.chunk_blocks = C;
   fp.item_prefix[0] = 0;
-  for (int r = 0; r < n; ++r) fp.item_prefix[r + 1] = fp.item_prefix[r] + ((nb[r] + C - 1) / C) * nkv;
+  for (int r = 0; r < n; ++r) {
+    fp.nch[r] = (nb[r] + C - 1) / C;
+    fp.item_prefix[r + 1] = fp.item_prefix[r] + fp.nch[r] * nkv;
+  }
   for (int r = n; r < kMaxBatch; ++r) fp.item_prefix[r + 1] = fp.item_prefix[n];
   fp.n_items = fp.item_prefix[n];
   if (fp.n_items > lay.f_max_items) return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "decode_step: split-KV scratch too small");
-  fp.H = sh.hidden, fp.nq = sh.n_q_heads, fp.nkv = nkv, fp.V = sh.vocab, fp.eps = sh.rms_eps;
-  fp.rope = m->w.rope_cos_sin;
-  fp.embed_q = m->w.embed.q, fp.embed_s = m->w.embed.scales, fp.embed_b = m->w.embed.biases;
   fp.pool = pool->mem;
   fp.layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
-  fp.x = at<uint16_t>(m, lay.x), fp.qkv = at<uint16_t>(m, lay.qkv), fp.attn = at<uint16_t>(m, lay.f_attn);
-  fp.ss = at<float>(m, lay.f_ss);
-  fp.pacc = at<float>(m, lay.f_pacc), fp.pml = at<float>(m, lay.f_pml);
-  fp.attn_counters = at<int>(m, lay.f_attn_counters), fp.amax = at<float2>(m, lay.f_amax);
   fp.next = next_dev, fp.logits = logits_dev;
-  fp.control = at<unsigned int>(m, lay.f_control);
   fp.timeline = m->timeline ? at<unsigned long long>(m, lay.f_timeline) : nullptr;
 
   auto launch = [&](int ph_begin, int ph_end, int from_x) -> int {
@@ -688,7 +693,7 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   m->last_h2d = m->last_d2h = 0;
   m->staging_next = 0;
   m->host_next = nullptr;
-  m->fused = false, m->fused_ctas = 0, m->timeline = false;
+  m->fused = false, m->fused_ctas = 0, m->timeline = false, m->fused_params = nullptr;
   m->host_status = nullptr, m->status_done = nullptr, m->status_pending = false;
   int dev = 0;
   cudaGetDevice(&dev);
@@ -706,20 +711,19 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   // Dense models run the whole step as one persistent kernel (Q4D_UNFUSED=1 selects the kernel-per-operation
   // sequence instead; mixture-of-experts models always use it).
   const char* unfused = getenv("Q4D_UNFUSED");
-  if (e == cudaSuccess && !shape->n_experts && !(unfused && unfused[0] == '1')) {
+  const bool narrow_gqa = shape->n_q_heads / shape->n_kv_heads <= 8;  // the whole-step kernel keeps 8 query heads per kv head
+  if (e == cudaSuccess && !shape->n_experts && narrow_gqa && !(unfused && unfused[0] == '1')) {
     int max_ctas = 0;
     e = fused_init(&max_ctas);
-    if (e == cudaSuccess && max_ctas > 0 && max_ctas <= lay.f_max_ctas) {
+    if (e == cudaSuccess && max_ctas > 0 && max_ctas <= lay.f_max_ctas && shape->n_layers <= kFusedMaxLayers) {
       m->fused = true;
       m->fused_ctas = max_ctas;
-      std::vector<FusedPhase> phases;
-      build_fused_phases(m, &phases);
-      for (int i = 0; i < kFusedDimKinds; ++i) {  // phase kinds: embedding, the phases of layer 0, final norm, LM head
-        const FusedPhase& P = phases[i < 8 ? i : phases.size() - 2 + (i - 8)];
-        FusedDims& D = m->fused_dims[i];
-        D.type = P.type, D.epi = P.epi, D.N = P.N, D.K = P.K, D.ntiles = P.ntiles, D.S = P.S, D.norm = P.norm, D.pad = 0;
+      m->fused_params = new (std::nothrow) FusedStep;
+      if (!m->fused_params) {
+        q4d_model_destroy(m);
+        return fail(Q4D_ERR_INVALID_ARG, "model_create: out of host memory");
       }
-      e = cudaMemcpy(m->ws + lay.f_phases, phases.data(), phases.size() * sizeof(FusedPhase), cudaMemcpyHostToDevice);
+      build_fused_params(m, m->fused_params);
       if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_attn_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
       if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_control, 0, 256);
       if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
@@ -743,6 +747,7 @@ int q4d_model_destroy(q4d_model* m) {
     if (m->staging_done[i]) cudaEventDestroy(m->staging_done[i]);
   }
   if (m->host_next) cudaFreeHost(m->host_next);
+  delete m->fused_params;
   if (m->host_status) cudaFreeHost(m->host_status);
   if (m->status_done) cudaEventDestroy(m->status_done);
   for (auto& r : m->prof_recs) cudaEventDestroy(r.a), cudaEventDestroy(r.b);
@@ -891,13 +896,11 @@ int q4d_timeline_read(q4d_model* m, float* us, int32_t* phases) {
   if (e != cudaSuccess) return fail_cuda(e, "timeline_read");
   const int np = m->lay.f_n_phases;
   std::vector<unsigned long long> stamps(np + 1);
-  std::vector<FusedPhase> table(np);
   e = cudaMemcpy(stamps.data(), m->ws + m->lay.f_timeline, stamps.size() * 8, cudaMemcpyDeviceToHost);
-  if (e == cudaSuccess) e = cudaMemcpy(table.data(), m->ws + m->lay.f_phases, table.size() * sizeof(FusedPhase), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return fail_cuda(e, "timeline_read");
   for (int i = 0; i < np; ++i) {
-    const int c = table[i].cls;
-    if (c < 0 || c >= Q4D_K_COUNT || stamps[i + 1] < stamps[i]) continue;
+    const int c = kFusedKindClass[fused_kind(i, np)];
+    if (stamps[i + 1] < stamps[i]) continue;
     us[c] += (float)((double)(stamps[i + 1] - stamps[i]) * 1e-3);
     phases[c] += 1;
   }

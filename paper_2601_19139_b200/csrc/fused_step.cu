@@ -37,21 +37,27 @@ namespace q4d {
 
 namespace {
 
-constexpr int kWarps = 8;
-constexpr int kDepth = 8;             // ring slots per warp (power of two)
+constexpr int kWarps = kFusedThreads / 32;
+constexpr int kDepth = 4;             // ring slots per warp (power of two)
 constexpr int kSlot = 2304;           // 16 rows x 128 B of codes (16-byte chunks XOR-swizzled) + 16 x (4 scales + 4 biases)
 constexpr int kSlotSb = 2048;         // offset of the scales/biases inside a slot
-constexpr int kActStride = 2 * kFusedSliceK + 16;  // bytes per request row of a staged slice (pad: no bank conflicts)
-constexpr int kActBytes = 16 * kActStride + (kFusedSliceK / 64) * 16 * 4;  // rows + group sums
+constexpr int kActRows = 16 * 2 * kFusedSliceK;     // bytes of a staged slice: 16 request rows, swizzled, no padding
+constexpr int kActBytes = kActRows + (kFusedSliceK / 64) * 16 * 4;  // rows + group sums
 constexpr int kRingBytes = kWarps * kDepth * kSlot;
-constexpr int kPartFloats = kWarps * 256;          // accumulators of the warps that share a tile
-constexpr int kMiscFloats = 16 + 256 + 128 + 128;  // inv, reduction scratch, argmax values, argmax indices
+constexpr int kPartFloats = (kWarps - kWarps / 4) * 256;  // accumulators of the warps that share a tile with a lead warp
+constexpr int kMiscFloats = 32 + 2 * kWarps * 16;  // reduction scratch, argmax values, argmax indices
 constexpr size_t kSmemBytes = (size_t)kRingBytes + 2 * kActBytes + (kPartFloats + kMiscFloats) * 4;
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
+  uint32_t r;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(r) : "r"(v));
+  return r;
+}
+
 constexpr float kScaleLog2 = 0.08838834764831845f * 1.4426950408889634f;  // log2(e) / sqrt(128)
 constexpr unsigned long long kBarrierTimeoutNs = 2000000000ull;
 
 static_assert((kDepth & (kDepth - 1)) == 0, "ring depth must be a power of two");
-static_assert(kDepth == 8, "the attention wait pattern assumes eight slots");
+static_assert(kDepth >= 4, "an attention block occupies four slots");
 static_assert(kFusedThreads == kWarps * 32, "thread count");
 static_assert(kSmemBytes <= 227 * 1024 - 256, "shared memory");
 
@@ -134,26 +140,52 @@ __device__ __forceinline__ int dims_index(const FusedStep& p, int ph) {
   return ph == 0 ? 0 : (ph >= p.n_phases - 2 ? 8 + (ph - (p.n_phases - 2)) : 1 + (ph - 1) % kFusedPhasesPerLayer);
 }
 __device__ __forceinline__ int phase_layer(int ph) { return (ph - 1) / kFusedPhasesPerLayer; }
+// Tensors of a projection phase (kind 2 QKV, 4 O, 6 gate/up, 7 down, 9 LM head), from the kernel parameters.
+struct GemmPtrs {
+  const uint32_t* qw;
+  const uint16_t* scales;
+  const uint16_t* biases;
+};
+__device__ __forceinline__ GemmPtrs gemm_ptrs(const FusedStep& p, int ph, int kind) {
+  GemmPtrs w;
+  if (kind == 9) {
+    w.qw = p.lm_qw, w.scales = p.lm_scales, w.biases = p.lm_biases;
+  } else {
+    const int j = kind == 2 ? 0 : (kind == 4 ? 1 : (kind == 6 ? 2 : 3));
+    const FusedLayerPtrs& L = p.layer[phase_layer(ph)];
+    w.qw = L.qw[j], w.scales = L.scales[j], w.biases = L.biases[j];
+  }
+  return w;
+}
 // Position of element e of a chunk of 8 in fragment order {0,4,1,5,2,6,3,7}.
 __device__ __forceinline__ int frag_pos(int e) { return (e & 3) * 2 + (e >> 2); }
 
-// A CTA's tiles are processed in groups: with five or more tiles left a warp owns a whole tile, with three or four
-// two warps share a tile (half of every slice each), with one or two four warps do.
-__device__ __forceinline__ void group_shape(int remaining, int& T_g, int& ksplit) {
-  if (remaining >= 5) {
-    T_g = remaining < 8 ? remaining : 8, ksplit = 1;
-  } else if (remaining >= 3) {
-    T_g = remaining, ksplit = 2;
+// A CTA's tiles are processed in groups: with more than half as many tiles left as the CTA has warps a warp owns
+// a whole tile, with more than a quarter two warps share a tile (half of every slice each), else four warps do.
+// (ksh = log2 of the number of warps per tile.)
+__device__ __forceinline__ void group_shape(int remaining, int& T_g, int& ksh) {
+  if (remaining > kWarps / 2) {
+    T_g = remaining < kWarps ? remaining : kWarps, ksh = 0;
+  } else if (remaining > kWarps / 4) {
+    T_g = remaining, ksh = 1;
   } else {
-    T_g = remaining, ksplit = 4;
+    T_g = remaining, ksh = 2;
   }
 }
-// The quads (256 input features) of slice s that belong to part pw of ksplit: first quad and count.
-__device__ __forceinline__ void my_quads(int K, int s, int ksplit, int pw, int& first, int& count) {
-  const int nqs = min(4, (K - s * kFusedSliceK) >> 8), qpp = 4 / ksplit;
+// The quads (256 input features) of slice s that belong to part pw of 1 << ksh: first quad and count.
+__device__ __forceinline__ void my_quads(int K, int s, int ksh, int pw, int& first, int& count) {
+  const int nqs = min(4, (K - s * kFusedSliceK) >> 8), qpp = 4 >> ksh;
   first = pw * qpp;
   const int c = nqs - first;
   count = c < 0 ? 0 : (c > qpp ? qpp : c);
+}
+// Where input feature k of request r sits in a projection's operand (K features), in elements.  The operand is
+// stored slice by slice (1024 features; all requests of a slice are contiguous, so one bulk copy stages a slice),
+// a request's slice as chunks of 8 features in MMA fragment order, and the 16-byte chunks of every 128 bytes
+// XOR-swizzled with the request index so that the fragment loads from shared memory are free of bank conflicts.
+__device__ __forceinline__ size_t operand_chunk(int K, int r, int k) {  // k a multiple of 8: offset of its chunk
+  const int k0 = k & ~(kFusedSliceK - 1), kw = min(kFusedSliceK, K - k0), chunk = (k - k0) >> 3;
+  return (size_t)16 * k0 + (size_t)r * kw + (size_t)((chunk ^ (r & 7)) << 3);
 }
 
 struct AttnItem {
@@ -165,41 +197,38 @@ __device__ __forceinline__ AttnItem decode_item(const FusedStep& p, int item) {
   while (r + 1 < p.n && item >= p.item_prefix[r + 1]) ++r;
   const int rem = item - p.item_prefix[r];
   it.r = r;
-  it.chunk = rem / p.nkv;
-  it.kvh = rem - it.chunk * p.nkv;
   it.T = p.lens[r] + 1;
   const int nb = (it.T + 15) >> 4;
-  it.nch = (nb + p.chunk_blocks - 1) / p.chunk_blocks;
+  it.nch = p.nch[r];
+  it.kvh = rem / it.nch;  // the chunks of a (request, kv head) are consecutive items
+  it.chunk = rem - it.kvh * it.nch;
   it.blk0 = it.chunk * p.chunk_blocks;
   it.nblk = min(p.chunk_blocks, nb - it.blk0);
   return it;
 }
 
 // Position of a warp's prefetch in its stream of ring stages (warp-uniform except the lane's source pointers).
+// The integer fields mean different things in projection and attention phases (a warp is in one at a time).
 struct IssueState {
   int ph, type;
-  // PH_GEMM: the walk over groups, slices and quads
-  int t_lo, T_c, done, T_g, ksplit, S, K, s, qi, q_first, q_count, rows_done;
-  const uint32_t* qw;
-  const uint16_t* scales;
-  const uint16_t* biases;
-  const uint32_t* qrow[4];  // this lane's four 16-byte chunks of the tile's rows, input feature 0
-  const uint16_t* sbrow;    // this lane's scale (lanes 0..15) or bias (16..31) row, group 0
-  // PH_ATTN
-  int item, st, nst, r, kvh, blk0, nblk, win;
-  const uint16_t* kbase;
+  int u[10];
+  const void* q[5];
 };
+// PH_GEMM: the walk over groups, slices and quads; q[0..3]: this lane's four 16-byte chunks of the tile's rows at
+// input feature 0; q[4]: this lane's scale (lanes 0..15) or bias (16..31) row at group 0
+enum { IG_TLO = 0, IG_TC, IG_DONE, IG_KSPLIT, IG_S, IG_K, IG_SLICE, IG_QI, IG_QFIRST, IG_QCOUNT };
+// PH_ATTN: the item and the stage within it; q[0]: K of the layer
+enum { IA_ITEM = 0, IA_ST, IA_NST, IA_R, IA_KVH, IA_BLK0, IA_NBLK };
 
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const FusedStep p) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ int s_abort;
   __shared__ __align__(8) uint64_t s_mbar[2];  // one per activation buffer
   unsigned char* acts = smem + kRingBytes;
-  float* s_part = reinterpret_cast<float*>(acts + 2 * kActBytes);  // [8 values][8 warps][32 lanes]
-  float* s_inv = s_part + kPartFloats;                             // [16]
-  float* s_red = s_inv + 16;                                       // [16][16]
-  float* s_bestv = s_red + 256;                                    // [8][16]
-  int* s_besti = reinterpret_cast<int*>(s_bestv + 128);            // [8][16]
+  float* s_part = reinterpret_cast<float*>(acts + 2 * kActBytes);  // [non-lead warp][8 values][32 lanes]
+  float* s_red = s_part + kPartFloats;                             // [warps]
+  float* s_bestv = s_red + 32;                                     // [warps][16]
+  int* s_besti = reinterpret_cast<int*>(s_bestv + kWarps * 16);    // [warps][16]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int cta = blockIdx.x, ncta = gridDim.x;
@@ -224,114 +253,115 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
   // ---------------------------------------------------------------- the issue side of the stage stream
   IssueState iss;
   iss.ph = p.ph_begin, iss.type = -1;
-  iss.t_lo = iss.T_c = iss.done = iss.T_g = iss.ksplit = iss.S = iss.K = iss.s = iss.qi = 0;
-  iss.q_first = iss.q_count = 0, iss.rows_done = -1;
-  iss.qw = nullptr, iss.scales = nullptr, iss.biases = nullptr, iss.sbrow = nullptr;
-  iss.qrow[0] = iss.qrow[1] = iss.qrow[2] = iss.qrow[3] = nullptr;
-  iss.item = iss.st = iss.nst = iss.r = iss.kvh = iss.blk0 = iss.nblk = iss.win = 0;
-  iss.kbase = nullptr;
+#pragma unroll
+  for (int i = 0; i < 10; ++i) iss.u[i] = 0;
+#pragma unroll
+  for (int i = 0; i < 5; ++i) iss.q[i] = nullptr;
   int islot = 0;
+  int win = 0, win_item = -1;  // window of block ids (blk0 + 32 * window + lane) of an attention item, and which item
 
-  // PH_GEMM: moves to the next (group, slice) at or after the current one in which this warp has quads.
-  auto iss_gemm_seek = [&]() -> bool {
+  // PH_GEMM: moves to the next (group, slice) at or after the current one in which this warp has quads; `fresh`
+  // says that the tile may have changed, so the lane's row pointers are loaded.
+  auto iss_gemm_seek = [&](bool fresh) -> bool {
     for (;;) {
-      if (iss.done >= iss.T_c) return false;
-      group_shape(iss.T_c - iss.done, iss.T_g, iss.ksplit);
-      const int tw = warp / iss.ksplit, pw = warp % iss.ksplit;
-      if (tw < iss.T_g) {
-        while (iss.s < iss.S) {
-          my_quads(iss.K, iss.s, iss.ksplit, pw, iss.q_first, iss.q_count);
-          if (iss.q_count > 0) break;
-          ++iss.s;
+      if (iss.u[IG_DONE] >= iss.u[IG_TC]) return false;
+      int T_g, ksh;
+      group_shape(iss.u[IG_TC] - iss.u[IG_DONE], T_g, ksh);
+      const int tw = warp >> ksh, pw = warp & ((1 << ksh) - 1);
+      if (tw < T_g) {
+        while (iss.u[IG_SLICE] < iss.u[IG_S]) {
+          my_quads(iss.u[IG_K], iss.u[IG_SLICE], ksh, pw, iss.u[IG_QFIRST], iss.u[IG_QCOUNT]);
+          if (iss.u[IG_QCOUNT] > 0) break;
+          ++iss.u[IG_SLICE];
         }
-        if (iss.s < iss.S) {
-          if (iss.rows_done != iss.done) {  // a new tile: this lane's row pointers
-            const FusedDims& D = p.dims[dims_index(p, iss.ph)];
-            const int tile = iss.t_lo + iss.done + tw;
+        if (iss.u[IG_SLICE] < iss.u[IG_S]) {
+          if (fresh) {
+            const int kind = dims_index(p, iss.ph);
+            const FusedDims& D = p.dims[kind];
+            const GemmPtrs P = gemm_ptrs(p, iss.ph, kind);
+            const int tile = iss.u[IG_TLO] + iss.u[IG_DONE] + tw, K = iss.u[IG_K];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
               const int row = unit_row(D.epi, D.N, tile, i * 4 + (lane >> 3));
-              iss.qrow[i] = iss.qw + (size_t)row * (iss.K >> 3) + (lane & 7) * 4;
+              iss.q[i] = P.qw + (size_t)row * (K >> 3) + (lane & 7) * 4;
             }
             const int row = unit_row(D.epi, D.N, tile, lane & 15);
-            iss.sbrow = (lane < 16 ? iss.scales : iss.biases) + (size_t)row * (iss.K >> 6);
-            iss.rows_done = iss.done;
+            iss.q[4] = (lane < 16 ? P.scales : P.biases) + (size_t)row * (K >> 6);
           }
           return true;
         }
       }
-      iss.done += iss.T_g;
-      iss.s = 0;
+      iss.u[IG_DONE] += T_g;
+      iss.u[IG_SLICE] = 0;
+      fresh = true;
     }
   };
   auto iss_attn_load = [&]() {
-    const AttnItem it = decode_item(p, iss.item);
-    iss.r = it.r, iss.kvh = it.kvh, iss.blk0 = it.blk0, iss.nblk = it.nblk;
-    iss.nst = 4 * it.nblk, iss.st = 0;
+    const AttnItem it = decode_item(p, iss.u[IA_ITEM]);
+    iss.u[IA_R] = it.r, iss.u[IA_KVH] = it.kvh, iss.u[IA_BLK0] = it.blk0, iss.u[IA_NBLK] = it.nblk;
+    iss.u[IA_NST] = 4 * it.nblk, iss.u[IA_ST] = 0;
   };
   auto iss_load_phase = [&]() {  // moves to the first phase at or after iss.ph in which this warp has stages
     while (iss.ph < p.ph_end) {
       const FusedDims& D = p.dims[dims_index(p, iss.ph)];
       iss.type = D.type;
       if (D.type == PH_GEMM) {
-        iss.t_lo = (int)((long long)cta * D.ntiles / ncta);
-        iss.T_c = (int)((long long)(cta + 1) * D.ntiles / ncta) - iss.t_lo;
-        iss.done = 0, iss.s = 0, iss.qi = 0, iss.S = D.S, iss.K = D.K, iss.rows_done = -1;
-        if (iss.T_c > 0) {
-          const FusedPhase& P = p.phases[iss.ph];
-          iss.qw = P.qw, iss.scales = P.scales, iss.biases = P.biases;
-          if (iss_gemm_seek()) break;
-        }
+        iss.u[IG_TLO] = (int)((long long)cta * D.ntiles / ncta);
+        iss.u[IG_TC] = (int)((long long)(cta + 1) * D.ntiles / ncta) - iss.u[IG_TLO];
+        iss.u[IG_DONE] = 0, iss.u[IG_SLICE] = 0, iss.u[IG_QI] = 0, iss.u[IG_S] = D.S, iss.u[IG_K] = D.K;
+        if (iss.u[IG_TC] > 0 && iss_gemm_seek(true)) break;
       } else if (D.type == PH_ATTN) {
-        iss.item = cta + ncta * warp;
-        if (iss.item < p.n_items) {
-          iss.kbase = p.pool + (size_t)(2 * phase_layer(iss.ph)) * p.layer_elems;
+        iss.u[IA_ITEM] = cta * kWarps + warp;
+        if (iss.u[IA_ITEM] < p.n_items) {
+          iss.q[0] = p.pool + (size_t)(2 * phase_layer(iss.ph)) * p.layer_elems;
           iss_attn_load();
           break;
         }
       }
       ++iss.ph;
     }
-    if (iss.ph + 1 < p.ph_end) prefetch_l1(p.phases + iss.ph + 1);
   };
   // Issues the next stage of the stream (if any) into the next ring slot and closes a cp.async group either way.
   auto issue_next = [&]() {
     if (iss.ph < p.ph_end) {
       unsigned char* stg = ring + islot * kSlot;
       if (iss.type == PH_GEMM) {
-        const int k = iss.s * kFusedSliceK + (iss.q_first + iss.qi) * 256;
+        const int k = iss.u[IG_SLICE] * kFusedSliceK + (iss.u[IG_QFIRST] + iss.u[IG_QI]) * 256;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int r = i * 4 + (lane >> 3);
-          cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), iss.qrow[i] + (k >> 3));
+          cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), static_cast<const uint32_t*>(iss.q[i]) + (k >> 3));
         }
-        cp_async8(stg + kSlotSb + (lane & 15) * 16 + (lane >> 4) * 8, iss.sbrow + (k >> 6));
-        if (++iss.qi == iss.q_count) {
-          iss.qi = 0;
-          ++iss.s;
-          if (!iss_gemm_seek()) {
+        cp_async8(stg + kSlotSb + (lane & 15) * 16 + (lane >> 4) * 8, static_cast<const uint16_t*>(iss.q[4]) + (k >> 6));
+        if (++iss.u[IG_QI] == iss.u[IG_QCOUNT]) {
+          iss.u[IG_QI] = 0;
+          ++iss.u[IG_SLICE];
+          if (!iss_gemm_seek(false)) {
             ++iss.ph;
             iss_load_phase();
           }
         }
       } else {
-        const int b = iss.st >> 2, part = iss.st & 3;
-        if (part == 0 && (b & 31) == 0) {
+        const int b = iss.u[IA_ST] >> 2, part = iss.u[IA_ST] & 3;
+        if (part == 0 && (b & 31) == 0 && (b != 0 || win_item != iss.u[IA_ITEM])) {
+          // block ids do not depend on the layer: the first window of an item is kept from one layer to the next
           const int idx = b + lane;
-          iss.win = idx < iss.nblk ? p.bt[(size_t)iss.r * p.max_blocks + iss.blk0 + idx] : 0;
+          win = idx < iss.u[IA_NBLK] ? p.bt[(size_t)iss.u[IA_R] * p.max_blocks + iss.u[IA_BLK0] + idx] : 0;
+          win_item = b == 0 ? iss.u[IA_ITEM] : -1;
         }
-        const int blk = __shfl_sync(0xffffffffu, iss.win, b & 31);
-        const uint16_t* base = (part < 2 ? iss.kbase : iss.kbase + p.layer_elems) +
-                               ((size_t)(blk * p.nkv + iss.kvh) * 16 + (part & 1) * 8) * kHeadDim;
+        const int blk = __shfl_sync(0xffffffffu, win, b & 31);
+        const uint16_t* kbase = static_cast<const uint16_t*>(iss.q[0]);
+        const uint16_t* base = (part < 2 ? kbase : kbase + p.layer_elems) +
+                               ((size_t)(blk * p.nkv + iss.u[IA_KVH]) * 16 + (part & 1) * 8) * kHeadDim;
         const unsigned char* src = reinterpret_cast<const unsigned char*>(base);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int c = i * 32 + lane, tok = c >> 4, c16 = c & 15;
           cp_async16(stg + tok * 256 + ((c16 ^ tok) << 4), src + c * 16);
         }
-        if (++iss.st == iss.nst) {
-          iss.item += ncta * kWarps;
-          if (iss.item < p.n_items) {
+        if (++iss.u[IA_ST] == iss.u[IA_NST]) {
+          iss.u[IA_ITEM] += ncta * kWarps;
+          if (iss.u[IA_ITEM] < p.n_items) {
             iss_attn_load();
           } else {
             ++iss.ph;
@@ -385,7 +415,6 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
 #pragma unroll 1
   for (int ph = p.ph_begin; ph < p.ph_end; ++ph) {
     const FusedDims& D = p.dims[dims_index(p, ph)];
-    if (ph + 1 < p.ph_end) prefetch_l1(p.phases + ph + 1);
 
     if (D.type == PH_EMBED) {
       // ---------------------------------------------------------- embedding (or sums of squares of a given x)
@@ -431,11 +460,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
     } else if (D.type == PH_NORM) {
       // ---------------------------------------------------------- RMSNorm: y = bf16(x / rms(x) * w), written once
       // for all CTAs as the operand of the next projection (chunks of 8 in fragment order)
-      const FusedPhase& P = p.phases[ph];
+      const int nkind = dims_index(p, ph);
+      const uint16_t* norm_w = nkind == 8 ? p.final_norm : p.layer[phase_layer(ph)].norm[nkind == 1 ? 0 : 1];
       const int H = D.K, cpr = H >> 3, total = p.n * cpr;
       const int lo = (int)((long long)cta * total / ncta), hi = (int)((long long)(cta + 1) * total / ncta);
       if (hi > lo) {
-        uint16_t* out = reinterpret_cast<uint16_t*>(P.out);
+        uint16_t* out = p.y;
         for (int r = lo / cpr; r <= (hi - 1) / cpr; ++r) {
           float sq = 0.0f;
           for (int j = threadIdx.x; j < (H >> 4); j += kFusedThreads) sq += __ldcg(p.ss + (size_t)j * 16 + r);
@@ -449,14 +479,14 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           const int c_lo = max(lo, r * cpr), c_hi = min(hi, (r + 1) * cpr);
           for (int c = c_lo + threadIdx.x; c < c_hi; c += kFusedThreads) {
             const int kc = c - r * cpr;
-            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(P.in + (size_t)r * H + kc * 8));
-            const uint4 wv = *reinterpret_cast<const uint4*>(P.norm_w + kc * 8);
+            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(p.x + (size_t)r * H + kc * 8));
+            const uint4 wv = *reinterpret_cast<const uint4*>(norm_w + kc * 8);
             const uint32_t e[4] = {v.x, v.y, v.z, v.w}, ww[4] = {wv.x, wv.y, wv.z, wv.w};
             uint32_t o[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               o[j] = pack_bf16x2(bf16_lo(e[j]) * inv * bf16_lo(ww[j]), bf16_hi(e[j]) * inv * bf16_hi(ww[j]));
-            *reinterpret_cast<uint4*>(out + (size_t)r * H + kc * 8) = permute_chunk(make_uint4(o[0], o[1], o[2], o[3]));
+            *reinterpret_cast<uint4*>(out + operand_chunk(H, r, kc * 8)) = permute_chunk(make_uint4(o[0], o[1], o[2], o[3]));
           }
           __syncthreads();
         }
@@ -466,34 +496,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
       const int t_lo = (int)((long long)cta * D.ntiles / ncta);
       const int T_c = (int)((long long)(cta + 1) * D.ntiles / ncta) - t_lo;
       if (T_c > 0) {
-        const FusedPhase& P = p.phases[ph];
-        const uint16_t* in = P.in;  // the operand as its producer wrote it: chunks of 8 in fragment order
+        // operand (as its producer wrote it) and output by kind: 2 QKV, 4 O, 6 gate/up, 7 down, 9 LM head
+        const int kind = dims_index(p, ph);
+        const uint16_t* in = kind == 4 ? p.attn : (kind == 7 ? p.h : p.y);
+        uint16_t* outp = kind == 2 ? p.qkv : (kind == 6 ? p.h : p.x);
+        const int out_stride = kind == 2 ? nqkv : p.H;
         const int K = D.K, S = D.S;
 
         // A slice of the operand goes to shared memory as one bulk copy per request row, tracked by the buffer's
         // mbarrier; the sums over every group of 64 input features come from the tensor cores (ones x operand).
         auto stage_issue = [&](int slice, int idx) {
-          if (threadIdx.x == 0) {
-            const int k0 = slice * kFusedSliceK, bytes = min(kFusedSliceK, K - k0) * 2;
-            unsigned char* dst = acts + (idx & 1) * kActBytes;
-            mbar_expect_tx(&s_mbar[idx & 1], (uint32_t)(bytes * p.n));
-            for (int r = 0; r < p.n; ++r)
-              bulk_copy_g2s(dst + r * kActStride, in + (size_t)r * K + k0, (uint32_t)bytes, &s_mbar[idx & 1]);
+          if (threadIdx.x == kFusedThreads - 32) {  // a lane of the last warp, which computes least often
+            const int k0 = slice * kFusedSliceK;
+            const uint32_t bytes = (uint32_t)(min(kFusedSliceK, K - k0) * 2 * p.n);  // rows 0..n-1 are contiguous
+            mbar_expect_tx(&s_mbar[idx & 1], bytes);
+            bulk_copy_g2s(acts + (idx & 1) * kActBytes, in + (size_t)16 * k0, bytes, &s_mbar[idx & 1]);
           }
+          // the other lanes of the issuing warp go on to spin on the mbarrier: they must not starve the issuing lane
+          __syncwarp();
         };
         auto stage_finish = [&](int slice, int idx) {
           if (!mbar_wait(&s_mbar[idx & 1], (uint32_t)((idx >> 1) & 1))) {
             if (lane == 0) atomicExch(p.control + 1, 2u);  // the copy never landed: report, results are void
           }
           const unsigned char* sB = acts + (idx & 1) * kActBytes;
-          float* sX = reinterpret_cast<float*>(acts + (idx & 1) * kActBytes + 16 * kActStride);
-          const int groups = min(kFusedSliceK, K - slice * kFusedSliceK) >> 6;
+          float* sX = reinterpret_cast<float*>(acts + (idx & 1) * kActBytes + kActRows);
+          const int kw2 = min(kFusedSliceK, K - slice * kFusedSliceK) * 2, groups = kw2 >> 7;
           const uint32_t one2 = 0x3F803F80u;  // bf16 {1, 1}
           for (int gi = warp; gi < groups; gi += kWarps) {
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt) {
-              const unsigned char* bp = sB + (nt * 8 + g) * kActStride + gi * 128 + t * 32;
-              const uint4 b0 = *reinterpret_cast<const uint4*>(bp), b1 = *reinterpret_cast<const uint4*>(bp + 16);
+              const unsigned char* row = sB + (nt * 8 + g) * kw2;
+              const uint4 b0 = *reinterpret_cast<const uint4*>(row + (((gi * 8 + t * 2) ^ g) << 4));
+              const uint4 b1 = *reinterpret_cast<const uint4*>(row + (((gi * 8 + t * 2 + 1) ^ g) << 4));
               float d[4];
               mma_bf16_first(d, one2, one2, one2, one2, b0.x, b0.y);
               mma_bf16(d, one2, one2, one2, one2, b0.z, b0.w);
@@ -504,48 +539,54 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           }
         };
 
-        // prologue: the first slice
-        stage_issue(0, staged);
-        stage_finish(0, staged);
+        // The CTA walks Q = groups x S slices; two of them are in flight at any time: slice q + 2 is requested as
+        // soon as slice q's buffer is free.
+        int n_groups = 0;
+        for (int d2 = 0; d2 < T_c; ++n_groups) {
+          int tg, kk;
+          group_shape(T_c - d2, tg, kk);
+          d2 += tg;
+        }
+        const int Q = n_groups * S, idx0 = staged;
+        staged += Q;
+        stage_issue(0, idx0);
+        if (Q > 1) stage_issue(1 % S, idx0 + 1);
+        stage_finish(0, idx0);
         __syncthreads();
-        int flat = staged++;  // index of the current slice's staging: buffer flat & 1
+        int q = 0;  // position in the walk: buffer (idx0 + q) & 1
 
         int done = 0;
 #pragma unroll 1
         while (done < T_c) {
-          int T_g, ksplit;
-          group_shape(T_c - done, T_g, ksplit);
-          const int tw = warp / ksplit, pw = warp % ksplit;
+          int T_g, ksh;
+          group_shape(T_c - done, T_g, ksh);
+          const int ksplit = 1 << ksh, tw = warp >> ksh, pw = warp & (ksplit - 1);
           const bool mine = tw < T_g, lead = mine && pw == 0;
           const int tile = t_lo + done + tw;
-          const bool more_groups = done + T_g < T_c;
           float acc[2][4];
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.0f;
           // the lead warp of a residual tile fetches the old values early
           uint16_t xold[8];
           if (lead && D.epi == EPI_RESIDUAL) {
-            const uint16_t* out = reinterpret_cast<const uint16_t*>(P.out);
+            const uint16_t* out = outp;
 #pragma unroll
             for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
               for (int c = 0; c < 4; ++c) {
                 const int req = nt * 8 + 2 * t + (c & 1), row = tile * 16 + g + (c >> 1) * 8;
-                xold[nt * 4 + c] = (req < p.n && row < D.N) ? __ldcg(out + (size_t)req * P.out_stride + row) : (uint16_t)0;
+                xold[nt * 4 + c] = (req < p.n && row < D.N) ? __ldcg(out + (size_t)req * out_stride + row) : (uint16_t)0;
               }
           }
 
 #pragma unroll 1
           for (int s = 0; s < S; ++s) {
-            const bool has_next = (s + 1 < S) || more_groups;
-            const int next_slice = (s + 1 < S) ? s + 1 : 0;
-            const int next_idx = staged;
-            if (has_next) stage_issue(next_slice, next_idx);
             if (mine) {
               int q_first, q_count;
-              my_quads(K, s, ksplit, pw, q_first, q_count);
-              const unsigned char* sB = acts + (flat & 1) * kActBytes;
-              const float* sX = reinterpret_cast<const float*>(sB + 16 * kActStride);
+              my_quads(K, s, ksh, pw, q_first, q_count);
+              const unsigned char* sB = acts + ((idx0 + q) & 1) * kActBytes;
+              const float* sX = reinterpret_cast<const float*>(sB + kActRows);
+              const int kw2 = min(kFusedSliceK, K - s * kFusedSliceK) * 2;  // bytes per request row of this slice
 #pragma unroll 1
               for (int qi = 0; qi < q_count; ++qi) {
                 const int qd = q_first + qi;
@@ -564,9 +605,9 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
                   float2 xs[2];
 #pragma unroll
                   for (int nt = 0; nt < 2; ++nt) {
-                    const unsigned char* bp = sB + (nt * 8 + g) * kActStride + gidx * 128 + t * 32;
-                    bf[nt][0] = *reinterpret_cast<const uint4*>(bp);
-                    bf[nt][1] = *reinterpret_cast<const uint4*>(bp + 16);
+                    const unsigned char* row = sB + (nt * 8 + g) * kw2;
+                    bf[nt][0] = *reinterpret_cast<const uint4*>(row + (((gidx * 8 + t * 2) ^ g) << 4));
+                    bf[nt][1] = *reinterpret_cast<const uint4*>(row + (((gidx * 8 + t * 2 + 1) ^ g) << 4));
                     xs[nt] = *reinterpret_cast<const float2*>(sX + gidx * 16 + nt * 8 + 2 * t);
                   }
                   const int off = (((gi * 2 + (t >> 1)) ^ g) << 4) + (t & 1) * 8;  // g: swizzle key of rows g, g + 8
@@ -597,40 +638,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
                 cslot = (cslot + 1) & (kDepth - 1);
               }
             }
-            if (has_next) {
-              stage_finish(next_slice, next_idx);
-              ++staged;
-            }
+            if (q + 1 < Q) stage_finish((q + 1) % S, idx0 + q + 1);
             __syncthreads();
-            flat = next_idx;
+            if (q + 2 < Q) stage_issue((q + 2) % S, idx0 + q + 2);
+            ++q;
           }
 
           // ---- warps that shared a tile: the lead warp adds the others' sums in warp order
           if (ksplit > 1) {
             if (mine && !lead) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) s_part[(i * kWarps + warp) * 32 + lane] = acc[i >> 2][i & 3];
+              for (int i = 0; i < 8; ++i) s_part[((warp - tw - 1) * 8 + i) * 32 + lane] = acc[i >> 2][i & 3];
             }
             __syncthreads();
             if (lead) {
               for (int o = 1; o < ksplit; ++o)
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[i >> 2][i & 3] += s_part[(i * kWarps + warp + o) * 32 + lane];
+                for (int i = 0; i < 8; ++i) acc[i >> 2][i & 3] += s_part[((warp + o - tw - 1) * 8 + i) * 32 + lane];
             }
           }
 
           // ---- epilogue: acc[nt][c]: row g + 8 * (c >> 1) of the tile, request nt * 8 + 2t + (c & 1)
           if (lead) {
             if (D.epi == EPI_SILU_PACK) {
-              uint16_t* out = reinterpret_cast<uint16_t*>(P.out);
-              const int col = tile * 8 + frag_pos(g);  // the tile's 8 columns are one chunk of the down projection's operand
+              uint16_t* out = outp;
+              // the tile's 8 columns are one chunk of the down projection's operand (N / 2 input features)
 #pragma unroll
               for (int nt = 0; nt < 2; ++nt)
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
                   const int req = nt * 8 + 2 * t + j;
                   const float gt = bf16_round(acc[nt][j]), up = bf16_round(acc[nt][2 + j]);
-                  if (req < p.n) out[(size_t)req * P.out_stride + col] = f32_to_bf16((gt / (1.0f + expf(-gt))) * up);
+                  if (req < p.n)
+                    out[operand_chunk(D.N >> 1, req, tile * 8) + frag_pos(g)] = f32_to_bf16((gt / (1.0f + expf(-gt))) * up);
                 }
             } else if (D.epi == EPI_F32) {
 #pragma unroll
@@ -646,7 +686,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
                   }
                 }
             } else {
-              uint16_t* out = reinterpret_cast<uint16_t*>(P.out);
+              uint16_t* out = outp;
               float sq[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
               for (int nt = 0; nt < 2; ++nt)
@@ -660,7 +700,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
                       const float f = bf16_to_f32(y);
                       sq[nt * 2 + (c & 1)] = fmaf(f, f, sq[nt * 2 + (c & 1)]);
                     }
-                    out[(size_t)req * P.out_stride + row] = y;
+                    out[(size_t)req * out_stride + row] = y;
                   }
                 }
               if (D.epi == EPI_RESIDUAL) {
@@ -712,30 +752,39 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
       }
     } else {
       // ---------------------------------------------------------- attention
-      const FusedPhase& P = p.phases[ph];
+      // Per 16-token block: S^T[token][head] = K q^T (tokens are the MMA rows, the G <= 8 query heads of the kv head
+      // the columns), online softmax down the columns, P^T transposed in registers (movmatrix) into the B operand of
+      // O^T[d][head] += V^T P^T with P split into two bf16 terms.
       const int layer = phase_layer(ph);
+      const FusedLayerPtrs& P = p.layer[layer];
       uint16_t* kpool_w = p.pool + (size_t)(2 * layer) * p.layer_elems;
+      const int Gs = (G + 1) & ~1;  // heads stored per partial result
+      // Items are dealt 16 consecutive ones to a CTA, one per warp, so the chunks of a (request, kv head) mostly meet
+      // in one CTA and are merged in shared memory (the activation buffers are idle during attention).
+      float* s_o = reinterpret_cast<float*>(acts);  // [warp][32 accumulator values][lane]
+      float* s_ml = s_part;                         // [warp][heads 2t, 2t+1 of t = 0..3][m, l]
+      const int per_round = ncta * kWarps;
 #pragma unroll 1
-      for (int item = cta + ncta * warp; item < p.n_items; item += ncta * kWarps) {
-        const AttnItem it = decode_item(p, item);
+      for (int base = cta * kWarps; base < p.n_items; base += per_round) {
+        const int item = base + warp;
+        const bool valid = item < p.n_items;
+        AttnItem it = decode_item(p, valid ? item : base);
         const int r = it.r, h = it.kvh, pos = it.T - 1;
+        if (!valid) it.nblk = 0;
         const uint16_t* qrow = p.qkv + (size_t)r * nqkv;
-        const bool appends = it.chunk == it.nch - 1;
+        const bool appends = valid && it.chunk == it.nch - 1;
 
-        // loads first: q of the G query heads, k and v of the new token, rotary table, block id of the append
-        uint32_t qa[8][4];
+        // loads first: q of head g, k and v of the new token, block id of the append
+        uint32_t qb[8][2];  // head g: dims 16ks + 2t, +1 and 16ks + 2t + 8, +9
         uint32_t wa = 0u, wb = 0u, nv_a = 0u, nv_b = 0u;
         int append_blk = 0;
         {
           const uint16_t* q0 = qrow + (size_t)(h * G + g) * kHeadDim;
-          const uint16_t* q1 = q0 + 8 * kHeadDim;
-          const bool v0 = g < G, v1 = g + 8 < G;
+          const bool v0 = g < G;
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            qa[ks][0] = v0 ? __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t)) : 0u;
-            qa[ks][1] = v1 ? __ldcg(reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t)) : 0u;
-            qa[ks][2] = v0 ? __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t + 8)) : 0u;
-            qa[ks][3] = v1 ? __ldcg(reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t + 8)) : 0u;
+            qb[ks][0] = v0 ? __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t)) : 0u;
+            qb[ks][1] = v0 ? __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t + 8)) : 0u;
           }
           if (appends) {
             const uint16_t* ksrc = qrow + (size_t)(p.nq + h) * kHeadDim;
@@ -747,48 +796,34 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
             append_blk = p.bt[(size_t)r * p.max_blocks + (pos >> 4)];
           }
         }
-        {
-          if (P.q_norm) {
-            float ss0 = 0.0f, ss1 = 0.0f;
+        if (P.q_norm) {
+          float ss = 0.0f;
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              ss0 += bf16_lo(qa[ks][0]) * bf16_lo(qa[ks][0]) + bf16_hi(qa[ks][0]) * bf16_hi(qa[ks][0]) +
-                     bf16_lo(qa[ks][2]) * bf16_lo(qa[ks][2]) + bf16_hi(qa[ks][2]) * bf16_hi(qa[ks][2]);
-              ss1 += bf16_lo(qa[ks][1]) * bf16_lo(qa[ks][1]) + bf16_hi(qa[ks][1]) * bf16_hi(qa[ks][1]) +
-                     bf16_lo(qa[ks][3]) * bf16_lo(qa[ks][3]) + bf16_hi(qa[ks][3]) * bf16_hi(qa[ks][3]);
-            }
-            ss0 += __shfl_xor_sync(0xffffffffu, ss0, 1);
-            ss0 += __shfl_xor_sync(0xffffffffu, ss0, 2);
-            ss1 += __shfl_xor_sync(0xffffffffu, ss1, 1);
-            ss1 += __shfl_xor_sync(0xffffffffu, ss1, 2);
-            const float inv0 = 1.0f / sqrtf(ss0 * (1.0f / kHeadDim) + p.eps);
-            const float inv1 = 1.0f / sqrtf(ss1 * (1.0f / kHeadDim) + p.eps);
+          for (int ks = 0; ks < 8; ++ks)
+            ss += bf16_lo(qb[ks][0]) * bf16_lo(qb[ks][0]) + bf16_hi(qb[ks][0]) * bf16_hi(qb[ks][0]) +
+                  bf16_lo(qb[ks][1]) * bf16_lo(qb[ks][1]) + bf16_hi(qb[ks][1]) * bf16_hi(qb[ks][1]);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+          const float inv = 1.0f / sqrtf(ss * (1.0f / kHeadDim) + p.eps);
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks)
-#pragma unroll
-              for (int rr = 0; rr < 4; ++rr) {
-                const int col = 16 * ks + 2 * t + (rr >> 1) * 8;
-                const uint32_t nw = *reinterpret_cast<const uint32_t*>(P.q_norm + col);
-                const float inv = (rr & 1) ? inv1 : inv0;
-                qa[ks][rr] = pack_bf16x2(bf16_lo(qa[ks][rr]) * inv * bf16_lo(nw), bf16_hi(qa[ks][rr]) * inv * bf16_hi(nw));
-              }
-          }
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
+          for (int ks = 0; ks < 8; ++ks)
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
-              const int col = 16 * ks + 2 * t + hf * 8;  // even, < 64
-              const float4 cs = *reinterpret_cast<const float4*>(p.rope + ((size_t)pos * 64 + col) * 2);  // c0 s0 c1 s1
-#pragma unroll
-              for (int rw = 0; rw < 2; ++rw) {
-                const int rr = hf * 2 + rw;
-                const float a0 = bf16_lo(qa[ks][rr]), a1 = bf16_hi(qa[ks][rr]);
-                const float b0 = bf16_lo(qa[ks + 4][rr]), b1 = bf16_hi(qa[ks + 4][rr]);
-                qa[ks][rr] = pack_bf16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
-                qa[ks + 4][rr] = pack_bf16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
-              }
+              const uint32_t nw = *reinterpret_cast<const uint32_t*>(P.q_norm + 16 * ks + 2 * t + hf * 8);
+              qb[ks][hf] = pack_bf16x2(bf16_lo(qb[ks][hf]) * inv * bf16_lo(nw), bf16_hi(qb[ks][hf]) * inv * bf16_hi(nw));
             }
         }
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const int col = 16 * ks + 2 * t + hf * 8;  // even, < 64
+            const float4 cs = *reinterpret_cast<const float4*>(p.rope + ((size_t)pos * 64 + col) * 2);  // c0 s0 c1 s1
+            const float a0 = bf16_lo(qb[ks][hf]), a1 = bf16_hi(qb[ks][hf]);
+            const float b0 = bf16_lo(qb[ks + 4][hf]), b1 = bf16_hi(qb[ks + 4][hf]);
+            qb[ks][hf] = pack_bf16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
+            qb[ks + 4][hf] = pack_bf16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
+          }
 
         // The warp with the request's last chunk prepares k, v of the new token and appends them to the pool.
         uint32_t nk_a = 0u, nk_b = 0u;  // elements 2*lane, 2*lane+1 and 64+2*lane, 64+2*lane+1
@@ -815,10 +850,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           *reinterpret_cast<uint32_t*>(vd + 64 + 2 * lane) = nv_b;
         }
 
-        float o[16][4];
+        // o[dt][c]: d = 16 dt + g + 8 (c >> 1), head 2t + (c & 1); m, l of heads 2t (index 0) and 2t + 1 (index 1)
+        float o[8][4];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
-        float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.0f, l_hi = 0.0f;
+        for (int j = 0; j < 8; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.0f;
+        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.0f, l1 = 0.0f;
 
 #pragma unroll 1
         for (int bi = 0; bi < it.nblk; ++bi) {
@@ -832,7 +868,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           unsigned char* sV0 = ring + ((cslot + 2) & (kDepth - 1)) * kSlot;
           unsigned char* sV1 = ring + ((cslot + 3) & (kDepth - 1)) * kSlot;
 
-          // K: eight stages are committed after this issue; the two K halves are the oldest two
+          // K: kDepth stages are committed after this issue; the two K halves are the oldest two
           issue_next();
           cp_async_wait<kDepth - 2>();
           __syncwarp();
@@ -842,19 +878,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
             *reinterpret_cast<uint32_t*>(kd + off_b) = nk_b;
             __syncwarp();
           }
-          // scores S[head][token] for the 16 tokens of the block
-          float s[2][4];
+          // scores: rows = tokens g, g + 8 of the block; columns = heads 2t, 2t + 1
+          float s[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+          {
+            const int mi = lane >> 3, tok = lane & 7;
+            const unsigned char* kb = ((mi & 1) ? sK1 : sK0) + tok * 256;
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const unsigned char* sK = j ? sK1 : sK0;
-            s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.0f;
-#pragma unroll
-            for (int kp = 0; kp < 4; ++kp) {
-              uint32_t kb[4];
-              const int tok = lane & 7, chunk = 4 * kp + (lane >> 3);
-              ldmatrix_x4(kb, sK + tok * 256 + ((chunk ^ tok) << 4));
-              mma_bf16(s[j], qa[2 * kp][0], qa[2 * kp][1], qa[2 * kp][2], qa[2 * kp][3], kb[0], kb[1]);
-              mma_bf16(s[j], qa[2 * kp + 1][0], qa[2 * kp + 1][1], qa[2 * kp + 1][2], qa[2 * kp + 1][3], kb[2], kb[3]);
+            for (int ks = 0; ks < 8; ++ks) {
+              uint32_t ka[4];
+              ldmatrix_x4(ka, kb + (((2 * ks + (mi >> 1)) ^ tok) << 4));
+              mma_bf16(s, ka[0], ka[1], ka[2], ka[3], qb[ks][0], qb[ks][1]);
             }
           }
           __syncwarp();
@@ -862,47 +895,44 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           issue_next();
           issue_next();
           if (tile * 16 + 16 > it.T) {  // ragged last block: tokens at or beyond T do not exist
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-              for (int c = 0; c < 4; ++c)
-                if (tile * 16 + 8 * j + 2 * t + (c & 1) >= it.T) s[j][c] = -INFINITY;
+            if (tile * 16 + g >= it.T) s[0] = s[1] = -INFINITY;
+            if (tile * 16 + g + 8 >= it.T) s[2] = s[3] = -INFINITY;
           }
 
-          // online softmax, rows g (lo) and g + 8 (hi); m is kept in log2 units
-          float mx_lo = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-          float mx_hi = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-          mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-          mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-          mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-          mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-          const float mn_lo = fmaxf(m_lo, mx_lo * kScaleLog2), mn_hi = fmaxf(m_hi, mx_hi * kScaleLog2);
-          const bool grow = (mn_lo > m_lo) || (mn_hi > m_hi);
+          // online softmax down the columns; m is kept in log2 units
+          float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
+#pragma unroll
+          for (int sh = 4; sh <= 16; sh <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, sh));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, sh));
+          }
+          const float mn0 = fmaxf(m0, mx0 * kScaleLog2), mn1 = fmaxf(m1, mx1 * kScaleLog2);
+          const bool grow = (mn0 > m0) || (mn1 > m1);
           if (__any_sync(0xffffffffu, grow)) {
-            const float c_lo = exp2f(m_lo - mn_lo), c_hi = exp2f(m_hi - mn_hi);
-            l_lo *= c_lo;
-            l_hi *= c_hi;
+            const float c0 = exp2f(m0 - mn0), c1 = exp2f(m1 - mn1);
+            l0 *= c0;
+            l1 *= c1;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              o[j][0] *= c_lo, o[j][1] *= c_lo;
-              o[j][2] *= c_hi, o[j][3] *= c_hi;
+            for (int j = 0; j < 8; ++j) {
+              o[j][0] *= c0, o[j][2] *= c0;
+              o[j][1] *= c1, o[j][3] *= c1;
             }
-            m_lo = mn_lo, m_hi = mn_hi;
+            m0 = mn0, m1 = mn1;
           }
-          uint32_t pH[4], pL[4];  // A fragments of P: hi and lo bf16 terms
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            const float p0 = exp2f(fmaf(s[j][0], kScaleLog2, -m_lo)), p1 = exp2f(fmaf(s[j][1], kScaleLog2, -m_lo));
-            const float p2 = exp2f(fmaf(s[j][2], kScaleLog2, -m_hi)), p3 = exp2f(fmaf(s[j][3], kScaleLog2, -m_hi));
-            l_lo += p0 + p1;
-            l_hi += p2 + p3;
-            const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
-            pH[2 * j] = h01, pH[2 * j + 1] = h23;
-            pL[2 * j] = pack_bf16x2(p0 - bf16_lo(h01), p1 - bf16_hi(h01));
-            pL[2 * j + 1] = pack_bf16x2(p2 - bf16_lo(h23), p3 - bf16_hi(h23));
+          uint32_t pH[2], pL[2];  // B fragments of P^T (head g; tokens 2t, 2t+1 and 2t+8, 2t+9): hi and lo bf16 terms
+          {
+            const float p0 = exp2f(fmaf(s[0], kScaleLog2, -m0)), p1 = exp2f(fmaf(s[1], kScaleLog2, -m1));
+            const float p2 = exp2f(fmaf(s[2], kScaleLog2, -m0)), p3 = exp2f(fmaf(s[3], kScaleLog2, -m1));
+            l0 += p0 + p2;
+            l1 += p1 + p3;
+            const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);  // (token g | g + 8; heads 2t, 2t+1)
+            const uint32_t e01 = pack_bf16x2(p0 - bf16_lo(h01), p1 - bf16_hi(h01));
+            const uint32_t e23 = pack_bf16x2(p2 - bf16_lo(h23), p3 - bf16_hi(h23));
+            pH[0] = movmatrix_trans(h01), pH[1] = movmatrix_trans(h23);
+            pL[0] = movmatrix_trans(e01), pL[1] = movmatrix_trans(e23);
           }
 
-          // V: ten stages are committed since the block began; the V halves are the third and fourth
+          // V: kDepth + 2 stages are committed since the block began; the V halves are the third and fourth
           cp_async_wait<kDepth - 2>();
           __syncwarp();
           if (patch) {
@@ -911,96 +941,165 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
             *reinterpret_cast<uint32_t*>(vd + off_b) = nv_b;
             __syncwarp();
           }
-          // O[head][d] += P[head][token] V[token][d]
+          // O^T[d][head] += V^T[d][token] P^T[token][head]
+          {
+            const int mi = lane >> 3, tok = lane & 7;
+            const unsigned char* vbase = ((mi >> 1) ? sV1 : sV0) + tok * 256;
 #pragma unroll
-          for (int jp = 0; jp < 8; ++jp) {
-            uint32_t vb[4];
-            const int i = lane >> 3, tok = lane & 7, chunk = 2 * jp + (i >> 1);
-            ldmatrix_x4_trans(vb, ((i & 1) ? sV1 : sV0) + tok * 256 + ((chunk ^ tok) << 4));
-            mma_bf16(o[2 * jp], pH[0], pH[1], pH[2], pH[3], vb[0], vb[1]);
-            mma_bf16(o[2 * jp], pL[0], pL[1], pL[2], pL[3], vb[0], vb[1]);
-            mma_bf16(o[2 * jp + 1], pH[0], pH[1], pH[2], pH[3], vb[2], vb[3]);
-            mma_bf16(o[2 * jp + 1], pL[0], pL[1], pL[2], pL[3], vb[2], vb[3]);
+            for (int dt = 0; dt < 8; ++dt) {
+              uint32_t va[4];
+              ldmatrix_x4_trans(va, vbase + (((2 * dt + (mi & 1)) ^ tok) << 4));
+              mma_bf16(o[dt], va[0], va[1], va[2], va[3], pH[0], pH[1]);
+              mma_bf16(o[dt], va[0], va[1], va[2], va[3], pL[0], pL[1]);
+            }
           }
           __syncwarp();
           cslot = (cslot + 4) & (kDepth - 1);
           issue_next();
         }
 
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-
-        uint16_t* arow = p.attn + (size_t)r * p.nq * kHeadDim + (size_t)h * G * kHeadDim;
-        if (it.nch == 1) {
-          const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
-          const int p0 = frag_pos(2 * t), p1 = frag_pos(2 * t + 1);  // chunk j of the head, elements 2t and 2t + 1
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            if (g < G) {
-              uint16_t* d = arow + (size_t)g * kHeadDim + 8 * j;
-              d[p0] = f32_to_bf16(o[j][0] * i_lo), d[p1] = f32_to_bf16(o[j][1] * i_lo);
-            }
-            if (g + 8 < G) {
-              uint16_t* d = arow + (size_t)(g + 8) * kHeadDim + 8 * j;
-              d[p0] = f32_to_bf16(o[j][2] * i_hi), d[p1] = f32_to_bf16(o[j][3] * i_hi);
-            }
-          }
-          continue;
+        for (int sh = 4; sh <= 16; sh <<= 1) {
+          l0 += __shfl_xor_sync(0xffffffffu, l0, sh);
+          l1 += __shfl_xor_sync(0xffffffffu, l1, sh);
         }
 
-        // publish the chunk's partial result; the last chunk to finish merges all of them in chunk order
-        {
-          float* pa = p.pacc + (size_t)item * G * kHeadDim;
-          float* pm = p.pml + (size_t)item * G * 2;
+        // ---- merge inside the CTA: every warp leaves its state in shared memory, the first warp of each run of
+        // chunks of one (request, kv head) adds the others' in chunk order
+        if (valid) {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            if (g < G) *reinterpret_cast<float2*>(pa + (size_t)g * kHeadDim + 8 * j + 2 * t) = make_float2(o[j][0], o[j][1]);
-            if (g + 8 < G)
-              *reinterpret_cast<float2*>(pa + (size_t)(g + 8) * kHeadDim + 8 * j + 2 * t) = make_float2(o[j][2], o[j][3]);
-          }
-          if (t == 0) {
-            if (g < G) *reinterpret_cast<float2*>(pm + g * 2) = make_float2(m_lo, l_lo);
-            if (g + 8 < G) *reinterpret_cast<float2*>(pm + (g + 8) * 2) = make_float2(m_hi, l_hi);
-          }
-          __syncwarp();
-          int last = 0;
-          if (lane == 0) {
-            __threadfence();  // the other lanes' stores, ordered before this by the warp barrier, become visible too
-            last = atom_acq_rel_add_s32(p.attn_counters + r * p.nkv + h, 1) == it.nch - 1;
-          }
-          last = __shfl_sync(0xffffffffu, last, 0);
-          if (!last) continue;
-          __threadfence();
-          const int item0 = p.item_prefix[r] + h;  // chunk c of this (request, kv head) is item0 + c * nkv
-          for (int a = 0; a < G; ++a) {
-            float M = -INFINITY;
-            for (int c = lane; c < it.nch; c += 32)
-              M = fmaxf(M, __ldcg(p.pml + ((size_t)(item0 + c * p.nkv) * G + a) * 2));
-#pragma unroll
-            for (int sh = 16; sh > 0; sh >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, sh));
-            float4 num = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            float den = 0.0f;
-#pragma unroll 4
-            for (int c = 0; c < it.nch; ++c) {
-              const size_t row = (size_t)(item0 + c * p.nkv) * G + a;
-              const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.pml + row * 2));
-              const float4 u = __ldcg(reinterpret_cast<const float4*>(p.pacc + row * kHeadDim + lane * 4));
-              const float e = exp2f(ml.x - M);
-              num.x = fmaf(e, u.x, num.x), num.y = fmaf(e, u.y, num.y);
-              num.z = fmaf(e, u.z, num.z), num.w = fmaf(e, u.w, num.w);
-              den = fmaf(e, ml.y, den);
-            }
-            // dims 4 * lane .. + 3: elements (lane & 1) * 4 .. + 3 of chunk lane >> 1
-            uint16_t* d = arow + (size_t)a * kHeadDim + (lane >> 1) * 8;
-            const int e0 = (lane & 1) * 4;
-            d[frag_pos(e0)] = f32_to_bf16(num.x / den), d[frag_pos(e0 + 1)] = f32_to_bf16(num.y / den);
-            d[frag_pos(e0 + 2)] = f32_to_bf16(num.z / den), d[frag_pos(e0 + 3)] = f32_to_bf16(num.w / den);
-          }
-          if (lane == 0) p.attn_counters[r * p.nkv + h] = 0;
+          for (int j = 0; j < 32; ++j) s_o[(warp * 32 + j) * 32 + lane] = o[j >> 2][j & 3];
+          if (g == 0) *reinterpret_cast<float4*>(s_ml + warp * 16 + 4 * t) = make_float4(m0, l0, m1, l1);
         }
+        __syncthreads();
+        if (valid && (it.chunk == 0 || warp == 0)) {
+          const int count = min(kWarps - warp, it.nch - it.chunk);
+          float M0 = m0, M1 = m1;
+          for (int w = 1; w < count; ++w) {
+            const float4 ml = *reinterpret_cast<const float4*>(s_ml + (warp + w) * 16 + 4 * t);
+            M0 = fmaxf(M0, ml.x), M1 = fmaxf(M1, ml.z);
+          }
+          {
+            const float c0 = exp2f(m0 - M0), c1 = exp2f(m1 - M1);
+            l0 *= c0, l1 *= c1;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              o[j][0] *= c0, o[j][2] *= c0;
+              o[j][1] *= c1, o[j][3] *= c1;
+            }
+          }
+          for (int w = 1; w < count; ++w) {
+            const float4 ml = *reinterpret_cast<const float4*>(s_ml + (warp + w) * 16 + 4 * t);
+            const float e0 = exp2f(ml.x - M0), e1 = exp2f(ml.z - M1);
+            l0 = fmaf(e0, ml.y, l0), l1 = fmaf(e1, ml.w, l1);
+            const float* so = s_o + (size_t)(warp + w) * 32 * 32 + lane;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              o[j][0] = fmaf(e0, so[(j * 4 + 0) * 32], o[j][0]);
+              o[j][1] = fmaf(e1, so[(j * 4 + 1) * 32], o[j][1]);
+              o[j][2] = fmaf(e0, so[(j * 4 + 2) * 32], o[j][2]);
+              o[j][3] = fmaf(e1, so[(j * 4 + 3) * 32], o[j][3]);
+            }
+          }
+
+          uint16_t* arow = p.attn;  // operand of the O projection: feature (h G + head) 128 + d of request r
+          const int Kq = p.nq * kHeadDim, feat0 = h * G * kHeadDim;
+          if (it.chunk == 0 && count == it.nch) {
+            // the whole (request, kv head): d = 16 dt + g (+ 8) is element g of chunk 2 dt (+ 1) of the head
+            const float i0 = 1.0f / l0, i1 = 1.0f / l1;
+            const int fp = frag_pos(g);
+#pragma unroll
+            for (int dt = 0; dt < 8; ++dt) {
+              if (2 * t < G) {
+                const int f = feat0 + (2 * t) * kHeadDim + 16 * dt;
+                arow[operand_chunk(Kq, r, f) + fp] = f32_to_bf16(o[dt][0] * i0);
+                arow[operand_chunk(Kq, r, f + 8) + fp] = f32_to_bf16(o[dt][2] * i0);
+              }
+              if (2 * t + 1 < G) {
+                const int f = feat0 + (2 * t + 1) * kHeadDim + 16 * dt;
+                arow[operand_chunk(Kq, r, f) + fp] = f32_to_bf16(o[dt][1] * i1);
+                arow[operand_chunk(Kq, r, f + 8) + fp] = f32_to_bf16(o[dt][3] * i1);
+              }
+            }
+          } else {
+            // the run is a part of the (request, kv head): publish it [d][Gs heads]; the last run to finish merges
+            float* pa = p.pacc + (size_t)item * kHeadDim * Gs;
+            float* pm = p.pml + (size_t)item * Gs * 2;
+            if (2 * t < Gs) {
+#pragma unroll
+              for (int dt = 0; dt < 8; ++dt) {
+                *reinterpret_cast<float2*>(pa + (size_t)(16 * dt + g) * Gs + 2 * t) = make_float2(o[dt][0], o[dt][1]);
+                *reinterpret_cast<float2*>(pa + (size_t)(16 * dt + g + 8) * Gs + 2 * t) = make_float2(o[dt][2], o[dt][3]);
+              }
+              if (g == 0) *reinterpret_cast<float4*>(pm + 4 * t) = make_float4(M0, l0, M1, l1);
+            }
+            __syncwarp();
+            const int i0 = item - it.chunk;  // first item of this (request, kv head)
+            const int runs = ((i0 + it.nch - 1) / kWarps) - (i0 / kWarps) + 1;
+            int last = 0;
+            if (lane == 0) {
+              __threadfence();  // the other lanes' stores, ordered before this by the warp barrier, become visible too
+              last = atom_acq_rel_add_s32(p.attn_counters + r * p.nkv + h, 1) == runs - 1;
+            }
+            last = __shfl_sync(0xffffffffu, last, 0);
+            if (last) {
+              __threadfence();
+              // lane: dims 4 lane .. 4 lane + 3, all heads; runs start at i0 and at every multiple of 16 after it
+              float M[8], den[8], num[4][8];
+#pragma unroll
+              for (int a = 0; a < 8; ++a) {
+                M[a] = -INFINITY, den[a] = 0.0f;
+                num[0][a] = num[1][a] = num[2][a] = num[3][a] = 0.0f;
+              }
+              for (int c = 0; c < runs; ++c) {
+                const int slot = c == 0 ? i0 : (i0 / kWarps + c) * kWarps;
+                const float* pmc = p.pml + (size_t)slot * Gs * 2;
+#pragma unroll
+                for (int a = 0; a < 8; ++a)
+                  if (a < Gs) M[a] = fmaxf(M[a], __ldcg(pmc + 2 * a));
+              }
+#pragma unroll 2
+              for (int c = 0; c < runs; ++c) {
+                const size_t slot = (size_t)(c == 0 ? i0 : (i0 / kWarps + c) * kWarps);
+                const float* pmc = p.pml + slot * Gs * 2;
+                const float* pac = p.pacc + slot * kHeadDim * Gs + (size_t)(4 * lane) * Gs;
+                float e[8];
+#pragma unroll
+                for (int a = 0; a < 8; ++a) {
+                  e[a] = 0.0f;
+                  if (a < Gs) {
+                    const float2 ml = __ldcg(reinterpret_cast<const float2*>(pmc + 2 * a));
+                    e[a] = exp2f(ml.x - M[a]);
+                    den[a] = fmaf(e[a], ml.y, den[a]);
+                  }
+                }
+#pragma unroll
+                for (int dd = 0; dd < 4; ++dd)
+#pragma unroll
+                  for (int a2 = 0; a2 < 4; ++a2)
+                    if (2 * a2 < Gs) {
+                      const float2 u = __ldcg(reinterpret_cast<const float2*>(pac + (size_t)dd * Gs + 2 * a2));
+                      num[dd][2 * a2] = fmaf(e[2 * a2], u.x, num[dd][2 * a2]);
+                      num[dd][2 * a2 + 1] = fmaf(e[2 * a2 + 1], u.y, num[dd][2 * a2 + 1]);
+                    }
+              }
+              // dims 4 lane .. + 3: elements (lane & 1) * 4 .. + 3 of chunk lane >> 1 of the head
+              const int e0 = (lane & 1) * 4;
+#pragma unroll
+              for (int a = 0; a < 8; ++a)
+                if (a < G) {
+                  uint16_t* d = arow + operand_chunk(Kq, r, feat0 + a * kHeadDim + (lane >> 1) * 8);
+#pragma unroll
+                  for (int dd = 0; dd < 4; ++dd) d[frag_pos(e0 + dd)] = f32_to_bf16(num[dd][a] / den[a]);
+                }
+              if (lane == 0) p.attn_counters[r * p.nkv + h] = 0;
+            }
+          }
+        }
+        __syncthreads();  // the next round reuses the shared-memory states
       }
+      // the activation buffers were written with ordinary stores; bulk copies (async proxy) write them next
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
 
     if (!grid_barrier(ph)) {

@@ -28,29 +28,23 @@ struct FusedDims {
   int pad;
 };
 
-// One phase of the step.  The table is built once per model and lives in device memory.
-struct alignas(128) FusedPhase {
-  int type;    // FusedPhaseType
-  int epi;     // PH_GEMM: GemmEpilogue
-  int N, K;    // PH_GEMM: output and input features
-  int ntiles;  // PH_GEMM: 16-row tiles (SiLU epilogue: 8 gate rows + the 8 matching up rows)
-  int S;       // PH_GEMM: K-slices of at most 1024 input features (the activations are staged slice by slice)
-  int norm;    // unused
-  int layer;   // PH_ATTN: layer of the pool
-  const uint32_t* qw;
-  const uint16_t* scales;
-  const uint16_t* biases;
-  const uint16_t* in;      // PH_GEMM: operand bf16 [16][K], chunks of 8 in fragment order; PH_NORM: x, plain
-  const uint16_t* norm_w;  // PH_NORM: bf16 [K]
-  void* out;               // PH_GEMM: output (bf16 [16][out_stride]; ignored for the f32 epilogue); PH_NORM: operand
-  const uint16_t* q_norm;  // PH_ATTN: bf16 [128] or NULL
+// Device pointers of one layer, by projection: 0 QKV, 1 O, 2 gate/up, 3 down.
+struct FusedLayerPtrs {
+  const uint32_t* qw[4];
+  const uint16_t* scales[4];
+  const uint16_t* biases[4];
+  const uint16_t* norm[2];  // attention norm, MLP norm
+  const uint16_t* q_norm;   // bf16 [128] or NULL
   const uint16_t* k_norm;
-  int out_stride;
-  int cls;                 // timeline class (Q4D_K_* of the unfused kernel this phase replaces)
 };
+constexpr int kFusedMaxLayers = 96;  // the pointers travel in the kernel parameters (constant bank: no loads on the way)
 
 struct FusedStep {
-  const FusedPhase* phases;
+  FusedLayerPtrs layer[kFusedMaxLayers];
+  const uint32_t* lm_qw;
+  const uint16_t* lm_scales;
+  const uint16_t* lm_biases;
+  const uint16_t* final_norm;
   FusedDims dims[kFusedDimKinds];  // by kind: 0 embedding, 1..7 the phases of a layer in order, 8 final norm, 9 LM head
   int n_phases;                    // phases of a whole step: 3 + 7 * layers
   int ph_begin, ph_end;
@@ -63,6 +57,7 @@ struct FusedStep {
   // attention plan: request r has ceil(blocks_r / chunk_blocks) chunks; items are (request, chunk, kv head)
   int chunk_blocks, n_items;
   int32_t item_prefix[17];
+  int32_t nch[16];  // chunks per (request, kv head)
   // shape
   int H, nq, nkv, V;
   float eps;
@@ -75,11 +70,13 @@ struct FusedStep {
   size_t layer_elems;
   // workspace
   uint16_t* x;      // residual stream bf16 [16][H]
+  uint16_t* y;      // normed hidden state, operand layout (K = H)
+  uint16_t* h;      // gated MLP activations, operand layout (K = mlp_inter)
   uint16_t* qkv;    // bf16 [16][(nq+2nkv)*128]
-  uint16_t* attn;   // attention output bf16 [16][nq*128], chunks of 8 in fragment order (operand of the O projection)
+  uint16_t* attn;   // attention output, operand layout (K = nq*128)
   float* ss;        // sums of squares of x: [H/16][16]
-  float* pacc;      // split-KV partial accumulators [item][G][128]
-  float* pml;       // [item][G][2] = (max in log2 units, sum)
+  float* pacc;      // split-KV partial accumulators [item][128][Gs], Gs = G rounded up to even
+  float* pml;       // [item][Gs][2] = (max in log2 units, sum)
   int* attn_counters;  // [16][nkv], zero between phases
   float2* amax;     // [ctas][16] (best logit, index bits)
   int32_t* next;    // [n]
@@ -88,7 +85,7 @@ struct FusedStep {
   unsigned long long* timeline;  // [phases + 1] nanosecond stamps, or NULL
 };
 
-constexpr int kFusedThreads = 256;
+constexpr int kFusedThreads = 512;
 constexpr int kFusedSliceK = 1024;
 
 size_t fused_smem_bytes();
