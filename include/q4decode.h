@@ -202,9 +202,10 @@ int q4d_profile_enable(q4d_model* model, int32_t on);
 int q4d_profile_read(q4d_model* model, float* ms, int32_t* launches);
 /* Kernel launches enqueued by this model since creation. */
 int64_t q4d_launch_count(q4d_model* model);
-/* 1 if the model runs a step as one persistent kernel (dense models; every phase of the step in one
- * cooperative launch, class Q4D_K_FUSED_STEP in the profile), 0 if it launches one kernel per operation
- * (mixture-of-experts models, or the environment variable Q4D_UNFUSED=1 at model creation). */
+/* 1 if the model runs a step as one persistent kernel (every phase of the step in one cooperative launch,
+ * class Q4D_K_FUSED_STEP in the profile), 0 if it launches one kernel per operation (the default).  The
+ * persistent kernel is chosen by the environment variable Q4D_STEP_KERNEL=fused at model creation and is
+ * available for dense models with at most 8 query heads per kv head and at most 96 layers. */
 int q4d_step_is_fused(q4d_model* model);
 /* Phase timeline of the persistent kernel.  While enabled, the kernel stamps the nanosecond clock after
  * every grid barrier.  q4d_timeline_read synchronises the device and adds up, for the most recent step,

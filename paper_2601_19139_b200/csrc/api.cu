@@ -63,7 +63,7 @@ struct Workspace {
   // x: residual stream (plain).  yp/ys, ap/as, hp/hs: GEMM operands in fragment order with their group sums
   // (normed hidden state, attention output, silu(gate)*up).
   size_t x, yp, ys, qkv, qbuf, ap, as, hp, hs, logits, next, amax, gemm_partial, gemm_partial_bytes, counters,
-      part_acc, part_ml, meta, bytes;
+      part_acc, part_ml, attn_merge_counters, meta, bytes;
   // MoE: plain normed state, routing results, touched-expert list, per-slot expert activations and outputs
   size_t yplain, m_idx, m_wgt, m_ints, m_hp, m_hs, m_o;
   int counters_len, amax_blocks;
@@ -171,6 +171,7 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   w.counters = take((size_t)cl * 4);
   w.part_acc = take((size_t)ml.max_work * s.n_q_heads * kHeadDim * 4);
   w.part_ml = take((size_t)ml.max_work * s.n_q_heads * 2 * 4);
+  w.attn_merge_counters = take((size_t)16 * s.n_kv_heads * 4);
   w.meta = take(ml.bytes);
   w.f_attn = w.f_h = w.f_ss = w.f_pacc = w.f_pml = w.f_attn_counters = w.f_amax = 0;
   w.f_control = w.f_timeline = 0;
@@ -572,8 +573,8 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     aa.n_work = plan.n_work, aa.n = n, aa.nq = nq, aa.nkv = nkv, aa.max_blocks = ml.max_blocks_cap;
     aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml);
     aa.out = nullptr, aa.out_xp = ap, aa.out_xs = as;
+    aa.merge_counters = at<int>(m, m->lay.attn_merge_counters);  // the last CTA of a (request, kv head) merges its chunks
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
-    Q4D_LAUNCH(Q4D_K_ATTN_MERGE, launch_attention_merge(aa, s));
     Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
     if (sh.n_experts == 0) {
       Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
@@ -706,13 +707,16 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   }
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_next), kMaxBatch * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
+  if (e == cudaSuccess) e = cudaMemset(m->ws + lay.attn_merge_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
   if (e == cudaSuccess && shape->n_experts)
     e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 2) * 4);
-  // Dense models run the whole step as one persistent kernel (Q4D_UNFUSED=1 selects the kernel-per-operation
-  // sequence instead; mixture-of-experts models always use it).
-  const char* unfused = getenv("Q4D_UNFUSED");
-  const bool narrow_gqa = shape->n_q_heads / shape->n_kv_heads <= 8;  // the whole-step kernel keeps 8 query heads per kv head
-  if (e == cudaSuccess && !shape->n_experts && narrow_gqa && !(unfused && unfused[0] == '1')) {
+  // The step runs as a chain of kernels (one per operation, programmatic dependent launches).  Dense models with at
+  // most 8 query heads per kv head can instead run the whole step as one persistent kernel: Q4D_STEP_KERNEL=fused at
+  // model creation.  On B200 the chain is the faster of the two, so it is the default.
+  const char* step_kernel = getenv("Q4D_STEP_KERNEL");
+  const bool want_fused = step_kernel && strcmp(step_kernel, "fused") == 0;
+  const bool narrow_gqa = shape->n_q_heads / shape->n_kv_heads <= 8;
+  if (e == cudaSuccess && want_fused && !shape->n_experts && narrow_gqa) {
     int max_ctas = 0;
     e = fused_init(&max_ctas);
     if (e == cudaSuccess && max_ctas > 0 && max_ctas <= lay.f_max_ctas && shape->n_layers <= kFusedMaxLayers) {

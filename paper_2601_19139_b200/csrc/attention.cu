@@ -30,6 +30,49 @@ constexpr int kTileBytes = 16 * 128 * 2;    // one block of one kv head: 16 toke
 constexpr int kAttnStage = 2 * kTileBytes;  // K then V
 constexpr float kScaleLog2 = 0.08838834764831845f * 1.4426950408889634f;  // log2(e) / sqrt(128)
 
+// out[r][a] = bf16(sum_c 2^(m_c - M) acc_c / sum_c 2^(m_c - M) l_c) over the request's chunks, in chunk order.
+// One call handles 8 consecutive elements (index ch of 16) of head a; the 8 lanes of an aligned lane group must hold
+// the 8 chunks of one 64-element group and all call together (group sums).  Writes the plain layout and/or the
+// fragment-ordered operand of the O projection (K = nq * 128) with its group sums.
+__device__ __forceinline__ void merge_head_chunk(const AttnArgs& p, int r, int a, int ch, bool valid) {
+  const int s0 = p.slot_base[r], nc = p.nchunks[r];
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float den = 0.0f;
+  if (valid) {
+    float M = -INFINITY;
+#pragma unroll 8
+    for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(p.part_ml + ((size_t)(s0 + c) * p.nq + a) * 2));
+#pragma unroll 4
+    for (int c = 0; c < nc; ++c) {
+      const size_t qh = (size_t)(s0 + c) * p.nq + a;
+      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + qh * 2));
+      const float4 u = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8));
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8 + 4));
+      const float e = exp2f(ml.x - M);
+      acc[0] = fmaf(e, u.x, acc[0]), acc[1] = fmaf(e, u.y, acc[1]), acc[2] = fmaf(e, u.z, acc[2]);
+      acc[3] = fmaf(e, u.w, acc[3]), acc[4] = fmaf(e, v.x, acc[4]), acc[5] = fmaf(e, v.y, acc[5]);
+      acc[6] = fmaf(e, v.z, acc[6]), acc[7] = fmaf(e, v.w, acc[7]);
+      den = fmaf(e, ml.y, den);
+    }
+  } else {
+    den = 1.0f;
+  }
+  uint4 o;
+  o.x = pack_bf16x2(acc[0] / den, acc[1] / den);
+  o.y = pack_bf16x2(acc[2] / den, acc[3] / den);
+  o.z = pack_bf16x2(acc[4] / den, acc[5] / den);
+  o.w = pack_bf16x2(acc[6] / den, acc[7] / den);
+  const float gsum = group_sum_8lanes(chunk_sum(o));  // 8 lanes = 64 elements = one group of the O projection's K
+  if (!valid) return;
+  const size_t col = (size_t)a * kHeadDim + ch * 8;
+  const size_t K = (size_t)p.nq * kHeadDim;
+  if (p.out) *reinterpret_cast<uint4*>(p.out + (size_t)r * K + col) = o;
+  if (p.out_xp) {
+    *reinterpret_cast<uint4*>(p.out_xp + (size_t)r * K + col) = permute_chunk(o);
+    if ((ch & 7) == 0) p.out_xs[(col >> 6) * 16 + r] = gsum;
+  }
+}
+
 __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const AttnArgs p) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -212,54 +255,35 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
         }
       }
     }
+    if (p.merge_counters) {
+      // the CTA that finishes the last chunk of this (request, kv head) merges all of them in chunk order
+      __shared__ int s_last;
+      __threadfence();
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        const int prev = atomicAdd(p.merge_counters + r * p.nkv + h, 1);
+        s_last = prev == p.nchunks[r] - 1;
+        if (s_last) p.merge_counters[r * p.nkv + h] = 0;
+      }
+      __syncthreads();
+      if (s_last) {
+        __threadfence();
+        for (int a0 = 0; a0 < G; a0 += 8) {  // 16 threads per head, 8 heads per pass
+          const int a = a0 + (threadIdx.x >> 4);
+          merge_head_chunk(p, r, h * G + a, threadIdx.x & 15, a < G);
+        }
+      }
+    }
     __syncthreads();
   }
 }
 
-// out[r][a] = bf16(sum_c 2^(m_c - M) acc_c / sum_c 2^(m_c - M) l_c) over the request's chunks, in chunk order.
-// 16 threads per head, 8 consecutive elements each; a CTA of 128 threads takes 8 heads.  Writes the plain
-// layout and/or the fragment-ordered operand of the O projection (K = nq * 128) with its group sums.
+// The merge as a kernel of its own: 16 threads per head; a CTA of 128 threads takes 8 heads.
 __global__ void __launch_bounds__(128) attention_merge_kernel(const AttnArgs p) {
   grid_launch_dependents();
   grid_dependency_wait();
   const int r = blockIdx.x, a = blockIdx.y * 8 + (threadIdx.x >> 4), ch = threadIdx.x & 15;
-  const bool valid = a < p.nq;
-  const int s0 = p.slot_base[r], nc = p.nchunks[r];
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  float den = 0.0f;
-  if (valid) {
-    float M = -INFINITY;
-#pragma unroll 8
-    for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(p.part_ml + ((size_t)(s0 + c) * p.nq + a) * 2));
-#pragma unroll 4
-    for (int c = 0; c < nc; ++c) {
-      const size_t qh = (size_t)(s0 + c) * p.nq + a;
-      const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + qh * 2));
-      const float4 u = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8));
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_acc + qh * kHeadDim + ch * 8 + 4));
-      const float e = exp2f(ml.x - M);
-      acc[0] = fmaf(e, u.x, acc[0]), acc[1] = fmaf(e, u.y, acc[1]), acc[2] = fmaf(e, u.z, acc[2]);
-      acc[3] = fmaf(e, u.w, acc[3]), acc[4] = fmaf(e, v.x, acc[4]), acc[5] = fmaf(e, v.y, acc[5]);
-      acc[6] = fmaf(e, v.z, acc[6]), acc[7] = fmaf(e, v.w, acc[7]);
-      den = fmaf(e, ml.y, den);
-    }
-  } else {
-    den = 1.0f;
-  }
-  uint4 o;
-  o.x = pack_bf16x2(acc[0] / den, acc[1] / den);
-  o.y = pack_bf16x2(acc[2] / den, acc[3] / den);
-  o.z = pack_bf16x2(acc[4] / den, acc[5] / den);
-  o.w = pack_bf16x2(acc[6] / den, acc[7] / den);
-  const float gsum = group_sum_8lanes(chunk_sum(o));  // 8 lanes = 64 elements = one group of the O projection's K
-  if (!valid) return;
-  const size_t col = (size_t)a * kHeadDim + ch * 8;
-  const size_t K = (size_t)p.nq * kHeadDim;
-  if (p.out) *reinterpret_cast<uint4*>(p.out + (size_t)r * K + col) = o;
-  if (p.out_xp) {
-    *reinterpret_cast<uint4*>(p.out_xp + (size_t)r * K + col) = permute_chunk(o);
-    if ((ch & 7) == 0) p.out_xs[(col >> 6) * 16 + r] = gsum;
-  }
+  merge_head_chunk(p, r, a, ch, a < p.nq);
 }
 
 // One warp per (request, head of qkv): optional RMSNorm over the head, rotary embedding at the

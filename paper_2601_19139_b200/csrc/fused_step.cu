@@ -44,7 +44,7 @@ constexpr int kSlotSb = 2048;         // offset of the scales/biases inside a sl
 constexpr int kActRows = 16 * 2 * kFusedSliceK;     // bytes of a staged slice: 16 request rows, swizzled, no padding
 constexpr int kActBytes = kActRows + (kFusedSliceK / 64) * 16 * 4;  // rows + group sums
 constexpr int kRingBytes = kWarps * kDepth * kSlot;
-constexpr int kPartFloats = (kWarps - kWarps / 4) * 256;  // accumulators of the warps that share a tile with a lead warp
+constexpr int kPartFloats = (kWarps - 2) * 256;  // accumulators of the warps that share a tile with a lead warp
 constexpr int kMiscFloats = 32 + 2 * kWarps * 16;  // reduction scratch, argmax values, argmax indices
 constexpr size_t kSmemBytes = (size_t)kRingBytes + 2 * kActBytes + (kPartFloats + kMiscFloats) * 4;
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t v) {
@@ -69,6 +69,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
 __device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned int ld_relaxed_u32(const unsigned int* p) {
+  unsigned int v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
 __device__ __forceinline__ void red_release_add_u32(unsigned int* p, unsigned int v) {
@@ -160,21 +165,30 @@ __device__ __forceinline__ GemmPtrs gemm_ptrs(const FusedStep& p, int ph, int ki
 // Position of element e of a chunk of 8 in fragment order {0,4,1,5,2,6,3,7}.
 __device__ __forceinline__ int frag_pos(int e) { return (e & 3) * 2 + (e >> 2); }
 
-// A CTA's tiles are processed in groups: with more than half as many tiles left as the CTA has warps a warp owns
-// a whole tile, with more than a quarter two warps share a tile (half of every slice each), else four warps do.
-// (ksh = log2 of the number of warps per tile.)
+// A CTA's tiles are processed in groups.  A group of T tiles gives every tile 16 / ceilpow2(T) warps, which split
+// the K range between them (ksh = log2 of the warps per tile; with 8 warps per tile a warp takes one quad of every
+// other slice).  The table picks the first group for a number of remaining tiles so that the chain of stages a warp
+// runs through is shortest, e.g. 11 tiles = 8 tiles x 2 warps, then 3 tiles x 4 warps.
+static_assert(kWarps == 16, "the group table is written for 16 warps");
 __device__ __forceinline__ void group_shape(int remaining, int& T_g, int& ksh) {
-  if (remaining > kWarps / 2) {
-    T_g = remaining < kWarps ? remaining : kWarps, ksh = 0;
-  } else if (remaining > kWarps / 4) {
-    T_g = remaining, ksh = 1;
+  if (remaining >= 16) {
+    T_g = 16, ksh = 0;
   } else {
-    T_g = remaining, ksh = 2;
+    // remaining:           1  2  3  4  5  6  7  8  9 10 11 12 13 14 15
+    const unsigned long long tg = 0xF88888887444321ull, ks = 0x011111111222233ull;
+    T_g = (int)((tg >> (4 * (remaining - 1))) & 0xF);
+    ksh = (int)((ks >> (4 * (remaining - 1))) & 0xF);
   }
 }
 // The quads (256 input features) of slice s that belong to part pw of 1 << ksh: first quad and count.
 __device__ __forceinline__ void my_quads(int K, int s, int ksh, int pw, int& first, int& count) {
-  const int nqs = min(4, (K - s * kFusedSliceK) >> 8), qpp = 4 >> ksh;
+  const int nqs = min(4, (K - s * kFusedSliceK) >> 8);
+  if (ksh == 3) {  // eight warps per tile: quad pw & 3 of the slices of parity pw >> 2
+    first = pw & 3;
+    count = ((s & 1) == (pw >> 2) && first < nqs) ? 1 : 0;
+    return;
+  }
+  const int qpp = 4 >> ksh;
   first = pw * qpp;
   const int c = nqs - first;
   count = c < 0 ? 0 : (c > qpp ? qpp : c);
@@ -224,6 +238,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ int s_abort;
   __shared__ __align__(8) uint64_t s_mbar[2];  // one per activation buffer
+  __shared__ int s_tlo[kFusedDimKinds], s_tc[kFusedDimKinds];  // this CTA's first tile and tile count by phase kind
   unsigned char* acts = smem + kRingBytes;
   float* s_part = reinterpret_cast<float*>(acts + 2 * kActBytes);  // [non-lead warp][8 values][32 lanes]
   float* s_red = s_part + kPartFloats;                             // [warps]
@@ -240,6 +255,11 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
   // one arrival (the thread that issues the bulk copies) per use.
   for (int i = threadIdx.x; i < 2 * kActBytes / 16; i += kFusedThreads)
     reinterpret_cast<uint4*>(acts)[i] = make_uint4(0u, 0u, 0u, 0u);
+  if (threadIdx.x < kFusedDimKinds) {
+    const int nt = p.dims[threadIdx.x].type == PH_GEMM ? p.dims[threadIdx.x].ntiles : 0;
+    s_tlo[threadIdx.x] = (int)((long long)cta * nt / ncta);
+    s_tc[threadIdx.x] = (int)((long long)(cta + 1) * nt / ncta) - s_tlo[threadIdx.x];
+  }
   if (threadIdx.x == 0) {
     s_abort = 0;
     mbar_init(&s_mbar[0], 1u);
@@ -303,11 +323,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
   };
   auto iss_load_phase = [&]() {  // moves to the first phase at or after iss.ph in which this warp has stages
     while (iss.ph < p.ph_end) {
-      const FusedDims& D = p.dims[dims_index(p, iss.ph)];
+      const int kind = dims_index(p, iss.ph);
+      const FusedDims& D = p.dims[kind];
       iss.type = D.type;
       if (D.type == PH_GEMM) {
-        iss.u[IG_TLO] = (int)((long long)cta * D.ntiles / ncta);
-        iss.u[IG_TC] = (int)((long long)(cta + 1) * D.ntiles / ncta) - iss.u[IG_TLO];
+        iss.u[IG_TLO] = s_tlo[kind];
+        iss.u[IG_TC] = s_tc[kind];
         iss.u[IG_DONE] = 0, iss.u[IG_SLICE] = 0, iss.u[IG_QI] = 0, iss.u[IG_S] = D.S, iss.u[IG_K] = D.K;
         if (iss.u[IG_TC] > 0 && iss_gemm_seek(true)) break;
       } else if (D.type == PH_ATTN) {
@@ -388,7 +409,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
       red_release_add_u32(p.control, 1u);
       const unsigned long long t0 = global_ns();
       unsigned int polls = 0;
-      while (ld_acquire_u32(p.control) < bar_target) {
+      while (ld_relaxed_u32(p.control) < bar_target) {
         if ((++polls & 63u) == 0) {
           if (ld_acquire_u32(p.control + 1) != 0u) {
             s_abort = 1;
@@ -401,6 +422,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
           }
         }
       }
+      asm volatile("fence.acq_rel.gpu;" ::: "memory");
       if (p.timeline && cta == 0) p.timeline[ph - p.ph_begin + 1] = global_ns();
     }
     __syncthreads();
@@ -493,8 +515,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_step_kernel(const Fuse
       }
     } else if (D.type == PH_GEMM) {
       // ---------------------------------------------------------- projection
-      const int t_lo = (int)((long long)cta * D.ntiles / ncta);
-      const int T_c = (int)((long long)(cta + 1) * D.ntiles / ncta) - t_lo;
+      const int t_lo = s_tlo[dims_index(p, ph)], T_c = s_tc[dims_index(p, ph)];
       if (T_c > 0) {
         // operand (as its producer wrote it) and output by kind: 2 QKV, 4 O, 6 gate/up, 7 down, 9 LM head
         const int kind = dims_index(p, ph);

@@ -88,6 +88,7 @@ struct AttnArgs {
   uint16_t* out;    // plain [n][nq][128], or NULL
   uint16_t* out_xp; // fragment-ordered operand [16][nq*128] of the O projection, or NULL
   float* out_xs;    // its group sums [nq*2][16]
+  int* merge_counters = nullptr;  // [16][nkv], zero between launches: the attention kernel merges the chunks itself
 };
 cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s);

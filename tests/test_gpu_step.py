@@ -43,6 +43,16 @@ def q4d():
     return binding
 
 
+@pytest.fixture(autouse=True, params=["chain", "fused"])
+def step_kernel(request, monkeypatch):
+    """Every test of this file runs twice: with the default chain of kernels and with the persistent whole-step
+    kernel (read from the environment when a model is created; models it does not support use the chain)."""
+    if request.param == "fused" and "moe" in request.node.name:
+        pytest.skip("mixture-of-experts models always use the chain of kernels")
+    monkeypatch.setenv("Q4D_STEP_KERNEL", request.param)
+    return request.param
+
+
 def _logit_err(g_logits, o_logits):
     """(max, rms) of the logit differences per request, in units of RMS(logits) of that request."""
     g, o = g_logits.astype(np.float64), o_logits.astype(np.float64)
