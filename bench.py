@@ -6,8 +6,8 @@ leaving and four joining (512 prefilled tokens) every 32 steps; `--workload` sel
 
   value      tokens/s with everything resident in HBM (tokens chained on the device, no host sync)
   e2e        tokens/s through q4d_decode_step_host: host inputs, host outputs, a sync per step
-  roofline   the dominant kernel (the persistent whole-step kernel of dense models) timed with CUDA events
-             around each of its launches
+  roofline   the dominant kernel (the launch class with the largest share of the step: a 4-bit projection or the
+             paged attention) timed with CUDA events around each of its launches
   cpu_baseline  the CPU oracle on a bounded sample of the same step, on the host cores
 
 `--impl reference` times the CPU oracle alone (the only reference implementation there is).
@@ -311,15 +311,31 @@ def main():
         tl_total = sum(v[0] for v in tl.values()) or 1.0
         kernels = {k: {"us_per_step": v[0], "phases_per_step": v[1], "share": v[0] / tl_total} for k, v in tl.items()}
     else:
+        # The dominant kernel is the launch class with the largest share of the step; its algorithmic bytes per
+        # launch are the packed tensor it streams (projections) or the cached K, V it reads (attention).
+        from workload import shapes as shp
+        H, d = shape.hidden, shape.head_dim
         kv_read_layer = float(np.mean([b["kv_read"] for b in bytes_log])) / shape.n_layers
-        att_ms, att_cnt = prof["attention"]
+        class_bytes = {"gemm_qkv": shp.q4_bytes(shape.qkv_out, H), "gemm_o": shp.q4_bytes(H, shape.n_q_heads * d),
+                       "gemm_gate_up": shp.q4_bytes(2 * shape.mlp_inter, H), "gemm_down": shp.q4_bytes(H, shape.mlp_inter),
+                       "lm_head": shp.q4_bytes(shape.vocab, H) + n * shape.vocab * 4, "attention": kv_read_layer}
+        class_kernel = {"attention": "paged_attention_kernel"}
+        # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped
+        # batch-16 case (see profiles/); traffic is proportional to the bytes streamed, so it is scaled to this launch.
+        traffic_ratio = {"gemm_gate_up": 1.005, "attention": 1.005}
         total_prof_ms = sum(v[0] for v in prof.values())
         kernels = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
                        "share": v[0] / total_prof_ms} for k, v in prof.items() if v[1]}
-        att_gbs = kv_read_layer / (att_ms / att_cnt * 1e-3) / 1e9 if att_cnt else 0.0
-        roofline = {"kernel": "paged_attention_kernel", "bound": "hbm", "achieved": att_gbs, "peak": peak,
-                    "unit": "GB/s", "frac": att_gbs / peak, "peak_kind": peak_kind, "traffic": None,
-                    "bytes_per_launch": kv_read_layer, "us_per_launch": att_ms / max(att_cnt, 1) * 1e3,
+        for k, v in kernels.items():
+            if k in class_bytes and prof[k][1]:
+                v["GBps"] = class_bytes[k] / (prof[k][0] / prof[k][1] * 1e-3) / 1e9
+        top = max((k for k in kernels if k in class_bytes), key=lambda k: kernels[k]["share"])
+        top_ms, top_cnt = prof[top]
+        gbs = class_bytes[top] / (top_ms / top_cnt * 1e-3) / 1e9
+        roofline = {"kernel": class_kernel.get(top, "q4_gemm_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
+                    "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": peak_kind,
+                    "traffic": class_bytes[top] * traffic_ratio[top] if top in traffic_ratio else None,
+                    "bytes_per_launch": float(class_bytes[top]), "us_per_launch": top_ms / top_cnt * 1e3,
                     "timing": "CUDA events around each launch, profile pass right after the timed steps"}
 
     # ---- max over ranks, aggregate ----
