@@ -560,11 +560,6 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     uint16_t* vpool = kpool + layer_elems;
     Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
     Q4D_LAUNCH(Q4D_K_GEMM_QKV, launch_q4_gemm(gemm_args(m, lw.wqkv, nqkv, H, yp, ys, n, EPI_BF16, qkv, nqkv), s));
-    RopeArgs ra;
-    ra.qkv = qkv, ra.q_norm = sh.qk_norm ? lw.q_norm : nullptr, ra.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
-    ra.eps = sh.rms_eps, ra.rope = m->w.rope_cos_sin, ra.n = n, ra.nq = nq, ra.nkv = nkv, ra.lens = d_lens;
-    ra.block_tables = d_bt, ra.max_blocks = ml.max_blocks_cap, ra.kpool = kpool, ra.vpool = vpool, ra.q_out = qbuf;
-    Q4D_LAUNCH(Q4D_K_ROPE_APPEND, launch_rope_append(ra, s));
     AttnArgs aa;
     aa.q = qbuf, aa.kpool = kpool, aa.vpool = vpool, aa.block_tables = d_bt, aa.lens = d_lens;
     aa.work = reinterpret_cast<const int4*>(dmeta + ml.off_work);
@@ -574,6 +569,9 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml);
     aa.out = nullptr, aa.out_xp = ap, aa.out_xs = as;
     aa.merge_counters = at<int>(m, m->lay.attn_merge_counters);  // the last CTA of a (request, kv head) merges its chunks
+    // q preparation (qk-norm, rotary embedding) and the append of k, v happen inside the attention kernel
+    aa.qkv = qkv, aa.q_norm = sh.qk_norm ? lw.q_norm : nullptr, aa.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
+    aa.eps = sh.rms_eps, aa.rope = m->w.rope_cos_sin, aa.kpool_w = kpool, aa.vpool_w = vpool;
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
     Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
     if (sh.n_experts == 0) {

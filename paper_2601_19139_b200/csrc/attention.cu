@@ -80,28 +80,16 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
   const int h = blockIdx.y;
 
   grid_launch_dependents();
-  grid_dependency_wait();
+  // The cached K, V, the lengths, the block tables and the work list are not written by the preceding kernel, so
+  // the first tiles are requested before it is awaited; q (and k, v of the new token) are read after the wait.
+  bool waited = false;
 
   for (int item = blockIdx.x; item < p.n_work; item += gridDim.x) {
     const int4 w = p.work[item];
     const int r = w.x, tile_begin = w.y, tile_end = w.z, slot = w.w;
-    const int T = p.lens[r] + 1;
+    const int T = p.lens[r] + 1, pos = T - 1;
     const int32_t* bt = p.block_tables + (size_t)r * p.max_blocks;
     unsigned char* ring = smem + warp * (kAttnStages * kAttnStage);
-
-    // Q fragments: rows = query heads of this kv head (zero beyond G), k = head dimension.
-    uint32_t qa[8][4];
-    {
-      const uint16_t* q0 = p.q + ((size_t)r * p.nq + (size_t)h * G + g) * kHeadDim;
-      const uint16_t* q1 = q0 + 8 * kHeadDim;
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t) : 0u;
-        qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t) : 0u;
-        qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t + 8) : 0u;
-        qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t + 8) : 0u;
-      }
-    }
 
     auto issue_tile = [&](int tile, int stage) {
       const int blk = bt[tile];
@@ -132,6 +120,104 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
       cp_async_commit();
     }
 
+    if (!waited) {
+      grid_dependency_wait();
+      waited = true;
+    }
+
+    // Q fragments: rows = query heads of this kv head (zero beyond G), k = head dimension.  With `qkv` given the
+    // kernel prepares q itself (per-head RMSNorm, rotary embedding at the request's position) and the CTA that holds
+    // the request's last tile also prepares k, v of the new token and appends them to the pool.
+    uint32_t qa[8][4];
+    const bool prep = p.qkv != nullptr;
+    {
+      const int heads = p.nq + 2 * p.nkv;
+      const uint16_t* qbase = prep ? p.qkv + (size_t)r * heads * kHeadDim : p.q + (size_t)r * p.nq * kHeadDim;
+      const uint16_t* q0 = qbase + (size_t)(h * G + g) * kHeadDim;
+      const uint16_t* q1 = q0 + 8 * kHeadDim;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qa[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t) : 0u;
+        qa[ks][1] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t) : 0u;
+        qa[ks][2] = (g < G) ? *reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 2 * t + 8) : 0u;
+        qa[ks][3] = (g + 8 < G) ? *reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 2 * t + 8) : 0u;
+      }
+    }
+    if (prep) {
+      if (p.q_norm) {
+        float ss0 = 0.0f, ss1 = 0.0f;  // rows g and g + 8
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          ss0 += bf16_lo(qa[ks][0]) * bf16_lo(qa[ks][0]) + bf16_hi(qa[ks][0]) * bf16_hi(qa[ks][0]) +
+                 bf16_lo(qa[ks][2]) * bf16_lo(qa[ks][2]) + bf16_hi(qa[ks][2]) * bf16_hi(qa[ks][2]);
+          ss1 += bf16_lo(qa[ks][1]) * bf16_lo(qa[ks][1]) + bf16_hi(qa[ks][1]) * bf16_hi(qa[ks][1]) +
+                 bf16_lo(qa[ks][3]) * bf16_lo(qa[ks][3]) + bf16_hi(qa[ks][3]) * bf16_hi(qa[ks][3]);
+        }
+        ss0 += __shfl_xor_sync(0xffffffffu, ss0, 1);
+        ss0 += __shfl_xor_sync(0xffffffffu, ss0, 2);
+        ss1 += __shfl_xor_sync(0xffffffffu, ss1, 1);
+        ss1 += __shfl_xor_sync(0xffffffffu, ss1, 2);
+        const float inv0 = 1.0f / sqrtf(ss0 * (1.0f / kHeadDim) + p.eps);
+        const float inv1 = 1.0f / sqrtf(ss1 * (1.0f / kHeadDim) + p.eps);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+#pragma unroll
+          for (int rr = 0; rr < 4; ++rr) {
+            const uint32_t nw = *reinterpret_cast<const uint32_t*>(p.q_norm + 16 * ks + 2 * t + (rr >> 1) * 8);
+            const float inv = (rr & 1) ? inv1 : inv0;
+            qa[ks][rr] = pack_bf16x2(bf16_lo(qa[ks][rr]) * inv * bf16_lo(nw), bf16_hi(qa[ks][rr]) * inv * bf16_hi(nw));
+          }
+      }
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int col = 16 * ks + 2 * t + hf * 8;  // even, < 64; its partner is col + 64 (k-step ks + 4)
+          const float4 cs = *reinterpret_cast<const float4*>(p.rope + ((size_t)pos * 64 + col) * 2);  // c0 s0 c1 s1
+#pragma unroll
+          for (int rw = 0; rw < 2; ++rw) {
+            const int rr = hf * 2 + rw;
+            const float a0 = bf16_lo(qa[ks][rr]), a1 = bf16_hi(qa[ks][rr]);
+            const float b0 = bf16_lo(qa[ks + 4][rr]), b1 = bf16_hi(qa[ks + 4][rr]);
+            qa[ks][rr] = pack_bf16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
+            qa[ks + 4][rr] = pack_bf16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
+          }
+        }
+    }
+    // k, v of the new token: the warp that walks the request's last tile prepares them, appends them to the pool and
+    // later puts them into its staged copy of that tile (which was fetched before they existed)
+    const int last_tile = pos >> 4;
+    const bool appends = prep && last_tile >= first && last_tile < tile_end && ((last_tile - first) % kAttnWarps) == 0;
+    uint32_t nk_a = 0u, nk_b = 0u, nv_a = 0u, nv_b = 0u;  // elements 2*lane, 2*lane+1 and 64+2*lane, 64+2*lane+1
+    if (appends) {
+      const int heads = p.nq + 2 * p.nkv;
+      const uint16_t* ksrc = p.qkv + ((size_t)r * heads + p.nq + h) * kHeadDim;
+      const uint16_t* vsrc = ksrc + (size_t)p.nkv * kHeadDim;
+      const uint32_t wa = *reinterpret_cast<const uint32_t*>(ksrc + 2 * lane);
+      const uint32_t wb = *reinterpret_cast<const uint32_t*>(ksrc + 64 + 2 * lane);
+      nv_a = *reinterpret_cast<const uint32_t*>(vsrc + 2 * lane);
+      nv_b = *reinterpret_cast<const uint32_t*>(vsrc + 64 + 2 * lane);
+      float a0 = bf16_lo(wa), a1 = bf16_hi(wa), b0 = bf16_lo(wb), b1 = bf16_hi(wb);
+      if (p.k_norm) {
+        const float ss = warp_sum(a0 * a0 + a1 * a1 + b0 * b0 + b1 * b1);
+        const float inv = 1.0f / sqrtf(ss * (1.0f / kHeadDim) + p.eps);
+        const uint32_t na = *reinterpret_cast<const uint32_t*>(p.k_norm + 2 * lane);
+        const uint32_t nb = *reinterpret_cast<const uint32_t*>(p.k_norm + 64 + 2 * lane);
+        a0 = bf16_to_f32(f32_to_bf16(a0 * inv * bf16_lo(na)));
+        a1 = bf16_to_f32(f32_to_bf16(a1 * inv * bf16_hi(na)));
+        b0 = bf16_to_f32(f32_to_bf16(b0 * inv * bf16_lo(nb)));
+        b1 = bf16_to_f32(f32_to_bf16(b1 * inv * bf16_hi(nb)));
+      }
+      const float4 cs = *reinterpret_cast<const float4*>(p.rope + ((size_t)pos * 64 + 2 * lane) * 2);
+      nk_a = pack_bf16x2(a0 * cs.x - b0 * cs.y, a1 * cs.z - b1 * cs.w);
+      nk_b = pack_bf16x2(b0 * cs.x + a0 * cs.y, b1 * cs.z + a1 * cs.w);
+      const size_t dst = (((size_t)bt[last_tile] * p.nkv + h) * kBlockSize + (pos & 15)) * kHeadDim;
+      *reinterpret_cast<uint32_t*>(p.kpool_w + dst + 2 * lane) = nk_a;
+      *reinterpret_cast<uint32_t*>(p.kpool_w + dst + 64 + 2 * lane) = nk_b;
+      *reinterpret_cast<uint32_t*>(p.vpool_w + dst + 2 * lane) = nv_a;
+      *reinterpret_cast<uint32_t*>(p.vpool_w + dst + 64 + 2 * lane) = nv_b;
+    }
+
     for (int it = 0; it < my_tiles; ++it) {
       const int tile = first + it * kAttnWarps;
       if (it + kAttnStages - 1 < my_tiles)
@@ -139,8 +225,18 @@ __global__ void __launch_bounds__(kAttnThreads) paged_attention_kernel(const Att
       cp_async_commit();
       cp_async_wait<kAttnStages - 1>();
       __syncwarp();
-      const unsigned char* sK = ring + (it % kAttnStages) * kAttnStage;
-      const unsigned char* sV = sK + kTileBytes;
+      unsigned char* sK = ring + (it % kAttnStages) * kAttnStage;
+      unsigned char* sV = sK + kTileBytes;
+      if (appends && tile == last_tile) {
+        const int tk = pos & 15;
+        const int off_a = tk * 256 + (((lane >> 2) ^ (tk & 7)) << 4) + (lane & 3) * 4;
+        const int off_b = tk * 256 + (((8 + (lane >> 2)) ^ (tk & 7)) << 4) + (lane & 3) * 4;
+        *reinterpret_cast<uint32_t*>(sK + off_a) = nk_a;
+        *reinterpret_cast<uint32_t*>(sK + off_b) = nk_b;
+        *reinterpret_cast<uint32_t*>(sV + off_a) = nv_a;
+        *reinterpret_cast<uint32_t*>(sV + off_b) = nv_b;
+        __syncwarp();
+      }
 
       // scores S[head][token] for the 16 tokens of the block
       float s[2][4];

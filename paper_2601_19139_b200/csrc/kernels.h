@@ -89,6 +89,15 @@ struct AttnArgs {
   uint16_t* out_xp; // fragment-ordered operand [16][nq*128] of the O projection, or NULL
   float* out_xs;    // its group sums [nq*2][16]
   int* merge_counters = nullptr;  // [16][nkv], zero between launches: the attention kernel merges the chunks itself
+  // With qkv given (bf16 [n][(nq+2nkv)*128], the QKV projection's output) the kernel prepares q itself (qk-norm,
+  // rotary embedding) and appends k, v of the new token to the pool; `q` is then unused.
+  const uint16_t* qkv = nullptr;
+  const uint16_t* q_norm = nullptr;  // bf16 [128] or NULL
+  const uint16_t* k_norm = nullptr;
+  float eps = 0.0f;
+  const float* rope = nullptr;  // f32 [positions][64][2]
+  uint16_t* kpool_w = nullptr;  // this layer of the pool, writable
+  uint16_t* vpool_w = nullptr;
 };
 cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s);
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s);
