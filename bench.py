@@ -34,6 +34,8 @@ WORKLOADS = {
     "qwen3-0.6b-b1": ("qwen3-0.6b-shaped", 1, 256, 256, False, False),
     "llama-3.2-3b-b16": ("llama-3.2-3b-shaped", 16, 512, 4096, False, False),
     "llama-3.2-3b-b1": ("llama-3.2-3b-shaped", 1, 512, 4096, False, False),
+    "moe-30b-b16": ("moe-30b-a3b-shaped", 16, 512, 4096, False, False),
+    "moe-30b-b1": ("moe-30b-a3b-shaped", 1, 512, 4096, False, False),
 }
 METRIC = "decode_tokens_per_second"
 
@@ -93,7 +95,12 @@ class ClockSampler:
 def step_bytes(shape, lens, n):
     """Algorithmic bytes of one step: packed weights + scales + biases, KV read and written, logits, embedding rows."""
     from workload import shapes
-    w = shapes.weight_bytes(shape)
+    # mixture of experts: the experts a step touches depend on the routing; the expectation under uniform routing
+    # (E * (1 - (1 - k/E)^n) distinct experts per layer) stands in for the count, which the library does not export
+    touched = None
+    if shape.n_experts:
+        touched = shape.n_experts * (1.0 - (1.0 - shape.top_k / shape.n_experts) ** n)
+    w = shapes.weight_bytes(shape, touched)
     per_tok_layer = 2 * shape.n_kv_heads * shape.head_dim * 2
     kv_read = int(sum(int(l) + 1 for l in lens)) * per_tok_layer * shape.n_layers
     kv_write = n * per_tok_layer * shape.n_layers
@@ -178,6 +185,9 @@ def main():
               "name": args.workload, "block_size": 16, "weights": "4-bit affine group-64, bf16 scale/bias",
               "l2": "inputs larger than L2 (weights + KV >> 126 MB); no flush needed",
               "layers": shape.n_layers, "hidden": shape.hidden, "vocab": shape.vocab}
+    if shape.n_experts:
+        config["experts"] = (f"{shape.n_experts} experts, top-{shape.top_k}; weight bytes count the expected number of "
+                             f"distinct experts per layer under uniform routing")
 
     if args.impl == "reference":
         # The reference arm is the CPU oracle: every "step" is the same bounded sample, extrapolated to a full step.
@@ -317,8 +327,13 @@ def main():
         H, d = shape.hidden, shape.head_dim
         kv_read_layer = float(np.mean([b["kv_read"] for b in bytes_log])) / shape.n_layers
         class_bytes = {"gemm_qkv": shp.q4_bytes(shape.qkv_out, H), "gemm_o": shp.q4_bytes(H, shape.n_q_heads * d),
-                       "gemm_gate_up": shp.q4_bytes(2 * shape.mlp_inter, H), "gemm_down": shp.q4_bytes(H, shape.mlp_inter),
+                       "gemm_gate_up": shp.q4_bytes(2 * shape.mlp_inter, H) if shape.mlp_inter else 0,
+                       "gemm_down": shp.q4_bytes(H, shape.mlp_inter) if shape.mlp_inter else 0,
                        "lm_head": shp.q4_bytes(shape.vocab, H) + n * shape.vocab * 4, "attention": kv_read_layer}
+        if shape.n_experts:  # expected distinct experts per layer (see step_bytes)
+            touched = shape.n_experts * (1.0 - (1.0 - shape.top_k / shape.n_experts) ** n)
+            class_bytes["moe_gate_up"] = touched * shp.q4_bytes(2 * shape.expert_inter, H)
+            class_bytes["moe_down"] = touched * shp.q4_bytes(H, shape.expert_inter)
         class_kernel = {"attention": "paged_attention_kernel"}
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped
         # batch-16 case (see profiles/); traffic is proportional to the bytes streamed, so it is scaled to this launch.
