@@ -69,7 +69,7 @@ struct Workspace {
   int counters_len, amax_blocks;
   // persistent whole-step kernel (dense models): plain attention output and gated MLP activations, sums of squares
   // of the residual stream, split-KV scratch, argmax partials, barrier/status words, phase table
-  size_t f_attn, f_h, f_ss, f_pacc, f_pml, f_attn_counters, f_amax, f_control, f_timeline;
+  size_t f_attn, f_h, f_ss, f_pacc, f_pml, f_attn_counters, f_amax, f_control, f_timeline, chain_status;
   int f_max_items, f_max_ctas, f_n_phases;
 };
 
@@ -150,7 +150,7 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   }
   w.logits = take(B * (size_t)s.vocab * 4);
   w.next = take(B * 4);
-  w.amax_blocks = (s.vocab + 127) / 128 + 1;
+  w.amax_blocks = std::max(gemm_row_blocks(s.vocab, s.hidden, 8, EPI_F32), gemm_row_blocks(s.vocab, s.hidden, 16, EPI_F32));
   w.amax = take((size_t)w.amax_blocks * 16 * sizeof(float2));
   size_t pb = 0;
   int cl = 0;
@@ -175,6 +175,7 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   w.meta = take(ml.bytes);
   w.f_attn = w.f_h = w.f_ss = w.f_pacc = w.f_pml = w.f_attn_counters = w.f_amax = 0;
   w.f_control = w.f_timeline = 0;
+  w.chain_status = take(256);  // status word of the chain's kernels (a bounded wait that gave up)
   w.f_max_items = w.f_max_ctas = w.f_n_phases = 0;
   if (!s.n_experts) {
     const int G = s.n_q_heads / s.n_kv_heads;
@@ -283,6 +284,7 @@ GemmArgs gemm_args(q4d_model* m, const q4d_qtensor& t, int N, int K, const uint1
   a.out_xp = nullptr, a.out_xs = nullptr, a.argmax_partial = nullptr;
   a.partial = at<float>(m, m->lay.gemm_partial), a.partial_bytes = m->lay.gemm_partial_bytes;
   a.counters = at<int>(m, m->lay.counters), a.counters_len = m->lay.counters_len;
+  a.status = at<unsigned int>(m, m->lay.chain_status);
   return a;
 }
 
@@ -346,7 +348,8 @@ void build_fused_params(const q4d_model* m, FusedStep* fp) {
   fp->control = reinterpret_cast<unsigned int*>(m->ws + lay.f_control);
 }
 
-// Reports a barrier timeout of an earlier step once its status word has come back.
+// Reports a wait that gave up inside a kernel of an earlier step (a grid barrier of the persistent kernel, a bulk
+// copy of the projection kernel) once the step's status word has come back.
 int fused_check_status(q4d_model* m, bool wait) {
   if (!m->status_pending) return Q4D_OK;
   cudaError_t e = wait ? cudaEventSynchronize(m->status_done) : cudaEventQuery(m->status_done);
@@ -354,7 +357,7 @@ int fused_check_status(q4d_model* m, bool wait) {
   if (e != cudaSuccess) return fail_cuda(e, "status read-back");
   m->status_pending = false;
   if (*m->host_status != 0u)
-    return fail(Q4D_ERR_TIMEOUT, "decode_step: a grid barrier of an earlier step timed out; destroy and re-create the model");
+    return fail(Q4D_ERR_TIMEOUT, "decode_step: a bounded wait inside a kernel of an earlier step gave up; destroy and re-create the model");
   return Q4D_OK;
 }
 
@@ -444,7 +447,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   if (!ids || !bt || max_blocks < 1 || (!range && ((!tokens_host && !tokens_dev) || !next_dev)))
     return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL argument");
   const q4d_shape& sh = m->sh;
-  if (m->fused) {
+  {
     const int rc = fused_check_status(m, false);
     if (rc != Q4D_OK) return rc;
   }
@@ -579,7 +582,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
       gu.out_xp = hp, gu.out_xs = hs;
       Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
-      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
+      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, nullptr, n, EPI_RESIDUAL, x, H), s));
     } else {
       const int E = sh.n_experts, Ie = sh.expert_inter;
       uint16_t* yplain = at<uint16_t>(m, m->lay.yplain);
@@ -621,6 +624,12 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   Q4D_LAUNCH(Q4D_K_LM_HEAD, launch_q4_gemm(lm, s));
   Q4D_LAUNCH(Q4D_K_ARGMAX, launch_argmax_finish(amax, lm_blocks, n, next_dev, s));
 #undef Q4D_LAUNCH
+  if (!m->status_pending) {
+    cudaError_t se = cudaMemcpyAsync(m->host_status, m->ws + m->lay.chain_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+    if (se == cudaSuccess) se = cudaEventRecord(m->status_done, s);
+    if (se != cudaSuccess) return fail_cuda(se, "status read-back");
+    m->status_pending = true;
+  }
 
   for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
   return Q4D_OK;
@@ -708,6 +717,10 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.attn_merge_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
   if (e == cudaSuccess && shape->n_experts)
     e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 2) * 4);
+  if (e == cudaSuccess) e = cudaMemset(m->ws + lay.chain_status, 0, 256);
+  if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->status_done, cudaEventDisableTiming);
+  if (e == cudaSuccess) *m->host_status = 0u;
   // The step runs as a chain of kernels (one per operation, programmatic dependent launches).  Dense models with at
   // most 8 query heads per kv head can instead run the whole step as one persistent kernel: Q4D_STEP_KERNEL=fused at
   // model creation.  On B200 the chain is the faster of the two, so it is the default.
@@ -728,9 +741,6 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
       build_fused_params(m, m->fused_params);
       if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_attn_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
       if (e == cudaSuccess) e = cudaMemset(m->ws + lay.f_control, 0, 256);
-      if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
-      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->status_done, cudaEventDisableTiming);
-      if (e == cudaSuccess) *m->host_status = 0u;
     }
   }
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -848,7 +858,7 @@ int q4d_decode_step_host(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64
     e = cudaMemcpyAsync(logits_host, d_logits, (size_t)n * m->sh.vocab * 4, cudaMemcpyDeviceToHost, s);
   if (e == cudaSuccess) e = cudaStreamSynchronize(s);
   if (e != cudaSuccess) return fail_cuda(e, "decode_step_host");
-  if (m->fused) {
+  {
     const int st = fused_check_status(m, true);
     if (st != Q4D_OK) return st;
   }

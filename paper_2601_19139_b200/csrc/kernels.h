@@ -46,6 +46,7 @@ struct GemmArgs {
   size_t partial_bytes;
   int* counters;  // zero between launches
   int counters_len;
+  unsigned int* status = nullptr;  // device word set non-zero when a bounded wait inside the kernel gives up
   // grouped mode (MoE): one GEMM per slot of a device-side list of touched experts; the tensors hold
   // `N` rows per expert, stacked.  NULL expert_ids = a single GEMM.
   const int* expert_ids = nullptr;  // [max_slots]

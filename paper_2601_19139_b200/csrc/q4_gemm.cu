@@ -10,16 +10,10 @@
 // no dequantised weight is ever rounded to bf16; scale and bias (less 16 * scale,
 // which removes the offset again) are applied to the fp32 group sums.
 //
-// Layout of the work.  A CTA of 8 warps owns 8*16*MT output rows and one
-// K-slice; each warp owns 16*MT rows and streams their packed codes, scales and
-// biases through a private cp.async ring in shared memory, 256 input features
-// (one "quad" of four groups, 128 B per row) per stage.  The activations arrive
-// already in MMA fragment order with their group sums (see common.cuh) and are
-// copied to shared memory asynchronously.  The weight stream does not depend on
-// the preceding kernel, so it is started before the grid dependency is awaited.
-// Split-K partial sums go to a scratch buffer; the last CTA to arrive for a row
-// block adds them in split order (the result does not depend on arrival order)
-// and applies the epilogue from a shared-memory tile.
+// Layout of the work: see q4_round_kernel below (one CTA per SM walks its row tiles in rounds, whole K or a part
+// of it inside the CTA; the weight stream does not depend on the preceding kernel, so it is started before the
+// grid dependency is awaited).  q4_gemm_kernel is the older CTA-granular form (a CTA owns 128 rows and one
+// K-slice, split-K through global scratch); the grouped mode of the mixture-of-experts layers still runs on it.
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -357,6 +351,502 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
   }
 }
 
+// ---- epilogue of a row tile ------------------------------------------------------------------------------------
+// Epilogue of one finished row tile from the accumulators in MMA fragment layout (lane holds rows g, g + 8 and
+// requests 2t, 2t + 1 of each block of 8 requests).  sE is 16 * (8 NT + 1) floats of the warp's own.
+template <int NT, class Params>
+__device__ __forceinline__ void tile_epilogue(const Params& p, const float (&acc)[NT][4], int tile, float* sE,
+                                              int lane, float& best, int& bidx) {
+  constexpr int NP = 8 * NT, kEs = NP + 1;
+  const int g = lane >> 2, t = lane & 3;
+  if (p.epilogue == EPI_SILU_PACK) {
+    // rows g are gate rows, rows g + 8 the matching up rows: h = bf16(silu(bf16(gate)) * bf16(up)) is lane-local
+    const int half_n = p.N >> 1;
+    uint16_t* sH = reinterpret_cast<uint16_t*>(sE);  // [NP][8]
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const float gt = bf16_to_f32(f32_to_bf16(acc[nt][j]));
+        const float up = bf16_to_f32(f32_to_bf16(acc[nt][2 + j]));
+        sH[(nt * 8 + 2 * t + j) * 8 + g] = f32_to_bf16((gt / (1.0f + expf(-gt))) * up);
+      }
+    __syncwarp();
+    const int col0 = tile * 8;
+    if (lane < NP && lane < p.n && col0 < half_n) {
+      const uint4 v = *reinterpret_cast<const uint4*>(sH + lane * 8);
+      *reinterpret_cast<uint4*>(p.out_xp + (size_t)lane * half_n + col0) = permute_chunk(v);
+    }
+    __syncwarp();
+    return;
+  }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) sE[(g + (c >> 1) * 8) * kEs + nt * 8 + 2 * t + (c & 1)] = acc[nt][c];
+  __syncwarp();
+  const int req = lane >> 1, half = lane & 1;
+  const int row0 = tile * 16 + half * 8;
+  float tb = -INFINITY;
+  int ti = 0x7fffffff;
+  if (req < NP && req < p.n && row0 < p.N) {
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = sE[(half * 8 + i) * kEs + req];
+    const bool full = row0 + 8 <= p.N && p.vec_ok;
+    if (p.epilogue == EPI_F32) {
+      float* o = reinterpret_cast<float*>(p.out) + (size_t)req * p.out_stride + row0;
+      if (full) {
+        *reinterpret_cast<float4*>(o) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(o + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (row0 + i < p.N) o[i] = v[i];
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if (row0 + i < p.N && v[i] > tb) tb = v[i], ti = row0 + i;  // ascending rows: the lowest row among equals
+    } else {
+      uint16_t* o = reinterpret_cast<uint16_t*>(p.out) + (size_t)req * p.out_stride + row0;
+      const bool res = p.epilogue == EPI_RESIDUAL;
+      if (full) {
+        uint4 old = make_uint4(0, 0, 0, 0);
+        if (res) old = *reinterpret_cast<const uint4*>(o);
+        const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+        uint32_t nw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float a = bf16_to_f32(f32_to_bf16(v[2 * i])), b = bf16_to_f32(f32_to_bf16(v[2 * i + 1]));
+          if (res) a += bf16_lo(ow[i]), b += bf16_hi(ow[i]);
+          nw[i] = pack_bf16x2(a, b);
+        }
+        *reinterpret_cast<uint4*>(o) = make_uint4(nw[0], nw[1], nw[2], nw[3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          if (row0 + i < p.N) {
+            uint16_t y = f32_to_bf16(v[i]);
+            if (res) y = f32_to_bf16(bf16_to_f32(o[i]) + bf16_to_f32(y));
+            o[i] = y;
+          }
+      }
+    }
+  }
+  if (p.epilogue == EPI_F32 && p.argmax_partial) {
+    // the two lanes of a request cover rows 0..7 and 8..15 of the tile; both keep the request's running best
+    const float ov = __shfl_xor_sync(0xffffffffu, tb, 1);
+    const int oi = __shfl_xor_sync(0xffffffffu, ti, 1);
+    if (ov > tb || (ov == tb && oi < ti)) tb = ov, ti = oi;
+    if (tb > best || (tb == best && ti < bidx)) best = tb, bidx = ti;
+  }
+  __syncwarp();
+}
+
+// ---- round kernel ------------------------------------------------------------------------------------------------
+// One CTA of 8 warps per SM owns a contiguous range of row tiles (MT sub-tiles of 16 rows each, so that the
+// activation fragments a warp reads from shared memory serve 16 MT rows: the multiply loop is bound by shared-memory
+// wavefronts, most of them activation reads) and one part of K (at most four slices of 1024 input features; most
+// projections have a single part).  It walks its tiles in rounds of at most 8 / kw tiles; kw warps share a tile
+// (stage j of the tile's stages goes to warp j mod kw of the tile) and add their accumulators through shared
+// memory at the end of the round.  The CTA moves through the slices together: the activations of the
+// next slice arrive by bulk copy in the other of two buffers while the warps multiply the current one, with one CTA
+// barrier per slice.  The weight rings (XOR-swizzled, no padding) run ahead across slices, tiles and rounds.  With
+// several parts of K the first warp of a tile hands its sums over through global scratch at the end of the round,
+// and the last part to arrive adds them in part order and applies the epilogue.
+struct RoundParams {
+  const uint32_t* qw;
+  const uint16_t* scales;
+  const uint16_t* biases;
+  const uint16_t* xp;
+  const float* xs;  // group sums of the operand, or NULL: the CTA adds them up itself
+  void* out;
+  uint16_t* out_xp;
+  float2* argmax_partial;  // [warps of the grid][16]
+  unsigned int* status;    // set to 3 when a wait gives up (may be NULL)
+  float* partial;          // [parts][T][MT * 16 * 8 NT] sums of a tile over one part of K (parts > 1 only)
+  int* counters;           // [T], zero between launches (parts > 1 only)
+  int N, K, n, out_stride, epilogue;
+  int T;   // row tiles of MT sub-tiles
+  int Tsub;  // sub-tiles of 16 rows (SiLU epilogue: 8 gate rows and the 8 matching up rows)
+  int Q;   // stages per K-slice
+  int S;   // K-slices per part; gridDim.y parts
+  int kw;  // warps per tile
+  int vec_ok;
+};
+
+#ifndef Q4D_ROUND_MT
+#define Q4D_ROUND_MT 1
+#endif
+constexpr int kRoundMT = Q4D_ROUND_MT;
+constexpr int kRoundWarps = 16 / kRoundMT, kRoundThreads = 32 * kRoundWarps;
+// a stage: 16 MT rows of 128 B of codes, 16-byte chunks swizzled by row, then the rows' scales and biases
+constexpr int kRoundRows = 16 * kRoundMT, kRoundStage = kRoundRows * (128 + kSbBytes);
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_g2s(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Waits for the phase with the given parity to complete; gives up (false) after a bounded number of tries.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (int tries = 0; tries < (1 << 17); ++tries) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
+template <int NT, int STAGES>
+__global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundParams p) {
+  constexpr int NP = 8 * NT, MT = kRoundMT, RW = kRoundRows;
+  constexpr int kEs = NP + 1;
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) uint64_t s_mbar[2];
+
+  grid_launch_dependents();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const bool silu = p.epilogue == EPI_SILU_PACK;
+  const int half_n = p.N >> 1;
+  const int Q = p.Q, S = p.S, SQ = S * Q, kw = p.kw;
+  const int parts = gridDim.y, part_j0 = blockIdx.y * SQ;  // this CTA's part of K starts at stage part_j0
+  const int ks = Q * 256;
+  const int b_stride = ks * 2 + 16;        // bytes per request row of a staged slice
+  const int act_bytes = NP * b_stride;     // one activation buffer
+  const int sum_bytes = Q * 4 * 16 * 4;    // group sums of a slice: [group][16]
+
+  unsigned char* ring = smem + warp * (STAGES * kRoundStage);
+  unsigned char* sAct = smem + kRoundWarps * STAGES * kRoundStage;  // two buffers
+  float* sSum = reinterpret_cast<float*>(sAct + 2 * act_bytes);     // two buffers
+  (void)kEs;
+
+  // the CTA's tiles and rounds
+  const int t0 = (int)((long long)blockIdx.x * p.T / gridDim.x), t1 = (int)((long long)(blockIdx.x + 1) * p.T / gridDim.x);
+  const int Tc = t1 - t0, tpr = kRoundWarps / kw;
+  const int R = (Tc + tpr - 1) / tpr;
+  const int base = R ? Tc / R : 0, rem = R ? Tc - base * R : 0;  // rounds [0, rem) hold base + 1 tiles
+  const int ts = warp / kw, kp = warp - ts * kw;
+  const int my_rounds = ts < base ? R : (ts == base ? rem : 0);  // the warp has a tile in rounds [0, my_rounds)
+  auto tile_of = [&](int r) -> int { return t0 + r * base + min(r, rem) + ts; };
+
+  // row r of a tile belongs to sub-tile tile * MT + r / 16
+  auto row_of = [&](int tile, int r) -> int {
+    const int sub = tile * MT + (r >> 4), rr = r & 15;
+    if (!silu) return min(sub * 16 + rr, p.N - 1);
+    return rr < 8 ? min(sub * 8 + rr, half_n - 1) : min(half_n + sub * 8 + (rr - 8), p.N - 1);
+  };
+  auto issue_stage = [&](int slot, int tile, int j) {
+    unsigned char* stg = ring + slot * kRoundStage;
+    const int kq = (part_j0 + j) * 256;
+#pragma unroll
+    for (int i = 0; i < RW / 4; ++i) {
+      const int r = i * 4 + (lane >> 3);
+      const int grow = row_of(tile, r);
+      const unsigned char* src =
+          reinterpret_cast<const unsigned char*>(p.qw + (size_t)grow * (p.K >> 3) + (kq >> 3)) + (lane & 7) * 16;
+      cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), src);
+    }
+    if (lane < RW) {
+      const int grow = row_of(tile, lane);
+      const size_t off = (size_t)grow * (p.K >> 6) + (kq >> 6);
+      cp_async8(stg + RW * 128 + lane * kSbBytes, p.scales + off);
+      cp_async8(stg + RW * 128 + lane * kSbBytes + 8, p.biases + off);
+    }
+  };
+
+  // cursors over the warp's stages: (round, stage of the tile), stage = kp, kp + kw, ...
+  int ir = 0, ij = kp;  // next stage to request
+  int cr = 0, cj = kp;  // next stage to multiply
+  int islot = 0, cslot = 0;
+  const bool any = my_rounds > 0 && kp < SQ;
+  // Weights do not depend on the preceding kernel: start streaming them before waiting for it.
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (any && ir < my_rounds) {
+      issue_stage(islot, tile_of(ir), ij);
+      ij += kw;
+      if (ij >= SQ) ij = kp, ++ir;
+      if (++islot == STAGES) islot = 0;
+    }
+    cp_async_commit();
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(&s_mbar[0], 1u);
+    mbar_init(&s_mbar[1], 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  grid_dependency_wait();
+
+  // One bulk copy per request row of the slice (and one for its group sums), tracked by the buffer's mbarrier.
+  auto stage_acts = [&](int gstep) {
+    if (threadIdx.x == 0) {
+      const int b = gstep & 1, slice = blockIdx.y * S + gstep % S;
+      const uint32_t bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
+      mbar_expect_tx(&s_mbar[b], bytes);
+      for (int r = 0; r < NP; ++r)
+        bulk_copy_g2s(sAct + b * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
+                      &s_mbar[b]);
+      if (p.xs) bulk_copy_g2s(sSum + b * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar[b]);
+    }
+    __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
+  };
+  const int steps = R * S;
+  if (steps > 0) stage_acts(0);
+
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0f;
+  float best = -INFINITY;
+  int bidx = 0x7fffffff;
+
+  int gstep = 0;
+  for (int r = 0; r < R; ++r) {
+    for (int s = 0; s < S; ++s, ++gstep) {
+      // the other buffer was last read in step gstep - 1, which every warp has left (barrier below)
+      if (gstep + 1 < steps) stage_acts(gstep + 1);
+      const int b = gstep & 1;
+      if (!mbar_wait(&s_mbar[b], (uint32_t)((gstep >> 1) & 1))) {
+        if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copy never landed: report, results are void
+      }
+      const unsigned char* sB = sAct + b * act_bytes;
+      float* sX = sSum + b * (sum_bytes / 4);
+      if (!p.xs) {
+        // the producer left no group sums: add up the 64 staged elements of every (group, request)
+        for (int c = threadIdx.x; c < Q * 4 * NP; c += kRoundThreads) {
+          const int gq = c / NP, rq = c - gq * NP;
+          const uint4* src = reinterpret_cast<const uint4*>(sB + rq * b_stride + gq * 128);
+          float sum = 0.0f;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) sum += chunk_sum(src[i]);
+          sX[gq * 16 + rq] = sum;
+        }
+        __syncthreads();
+      }
+
+      while (any && cr == r && cr < my_rounds && cj < (s + 1) * Q) {
+        if (ir < my_rounds) {
+          issue_stage(islot, tile_of(ir), ij);
+          ij += kw;
+          if (ij >= SQ) ij = kp, ++ir;
+          if (++islot == STAGES) islot = 0;
+        }
+        cp_async_commit();
+        cp_async_wait<STAGES - 1>();
+        __syncwarp();
+        const unsigned char* stg = ring + cslot * kRoundStage;
+        if (++cslot == STAGES) cslot = 0;
+        const int cq = cj - s * Q;
+
+        uint2 sc[MT][2], bi[MT][2];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint4 v = *reinterpret_cast<const uint4*>(stg + RW * 128 + (mt * 16 + g + 8 * h) * kSbBytes);
+            sc[mt][h] = make_uint2(v.x, v.y);
+            bi[mt][h] = make_uint2(v.z, v.w);
+          }
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) {
+          const int gidx = cq * 4 + gi;
+          uint4 bf[NT][2];
+          float2 xs[NT];
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const unsigned char* bp = sB + (nt * 8 + g) * b_stride + gidx * 128 + t * 32;
+            bf[nt][0] = *reinterpret_cast<const uint4*>(bp);
+            bf[nt][1] = *reinterpret_cast<const uint4*>(bp + 16);
+            xs[nt] = *reinterpret_cast<const float2*>(sX + gidx * 16 + nt * 8 + 2 * t);
+          }
+          // 16-byte chunk c of row r sits at chunk c ^ (r & 7); rows g, g + 8, g + 16, ... share the swizzle
+          const int woff = g * 128 + (((gi * 2 + (t >> 1)) ^ g) << 4) + (t & 1) * 8;
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const uint2 wl = *reinterpret_cast<const uint2*>(stg + mt * 16 * 128 + woff);
+            const uint2 wh = *reinterpret_cast<const uint2*>(stg + mt * 16 * 128 + woff + 8 * 128);
+            uint32_t l0[4], l1[4], h0[4], h1[4];
+            unpack_word(wl.x, l0);
+            unpack_word(wl.y, l1);
+            unpack_word(wh.x, h0);
+            unpack_word(wh.y, h1);
+            // sum (16 + q) x = 16 X + sum q x, so the bias that multiplies X becomes b - 16 s
+            const float s_lo = bf16_at(sc[mt][0], gi), s_hi = bf16_at(sc[mt][1], gi);
+            const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[mt][0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[mt][1], gi));
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              float pc[4];
+              mma_bf16_first(pc, l0[0], h0[0], l0[1], h0[1], bf[nt][0].x, bf[nt][0].y);
+              mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
+              mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
+              mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
+              acc[mt][nt][0] = fmaf(s_lo, pc[0], fmaf(b_lo, xs[nt].x, acc[mt][nt][0]));
+              acc[mt][nt][1] = fmaf(s_lo, pc[1], fmaf(b_lo, xs[nt].y, acc[mt][nt][1]));
+              acc[mt][nt][2] = fmaf(s_hi, pc[2], fmaf(b_hi, xs[nt].x, acc[mt][nt][2]));
+              acc[mt][nt][3] = fmaf(s_hi, pc[3], fmaf(b_hi, xs[nt].y, acc[mt][nt][3]));
+            }
+          }
+        }
+        __syncwarp();
+        cj += kw;
+        if (cj >= SQ) cj = kp, ++cr;
+      }
+
+      if (s == S - 1 && kw > 1 && kp != 0 && r < my_rounds) {
+        // hand the accumulators to the tile's first warp through the ring slot this warp has just multiplied: it
+        // is free until the warp requests its next stage (lane-major: conflict-free both ways)
+        float4* dst = reinterpret_cast<float4*>(ring + (cslot == 0 ? STAGES - 1 : cslot - 1) * kRoundStage);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            dst[(mt * NT + nt) * 32 + lane] = make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
+      }
+      __syncthreads();
+    }
+    // round end: the first warp of every tile adds its partners in warp order and applies the epilogue
+    if (r < my_rounds && kp == 0) {
+      for (int k = 1; k < kw; ++k) {
+        // partner k has multiplied (r + 1) * ceil((SQ - k) / kw) stages so far: its last slot follows from that
+        const int pslot = ((r + 1) * ((SQ - k + kw - 1) / kw) - 1) % STAGES;
+        const float4* src = reinterpret_cast<const float4*>(smem + (warp + k) * (STAGES * kRoundStage) + pslot * kRoundStage);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const float4 a = src[(mt * NT + nt) * 32 + lane];
+            acc[mt][nt][0] += a.x, acc[mt][nt][1] += a.y, acc[mt][nt][2] += a.z, acc[mt][nt][3] += a.w;
+          }
+      }
+      const int tile = tile_of(r);
+      bool finish = true;
+      if (parts > 1) {
+        // several CTAs hold parts of this tile's sums: publish, and the last to arrive adds them in part order
+        constexpr int kF4 = 32 * MT * NT;  // float4 per tile and part
+        float4* part = reinterpret_cast<float4*>(p.partial) + ((size_t)blockIdx.y * p.T + tile) * kF4;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            part[(mt * NT + nt) * 32 + lane] = make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
+        __threadfence();
+        __syncwarp();
+        int prev = 0;
+        if (lane == 0) prev = atomicAdd(p.counters + tile, 1);
+        prev = __shfl_sync(0xffffffffu, prev, 0);
+        finish = prev == parts - 1;
+        if (finish) {
+          __threadfence();
+          if (lane == 0) p.counters[tile] = 0;
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+              for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0f;
+          for (int y0 = 0; y0 < parts; y0 += 2) {  // two parts at a time: their loads go out together
+            float4 v[2][MT * NT];
+#pragma unroll
+            for (int y = 0; y < 2; ++y)
+#pragma unroll
+              for (int i = 0; i < MT * NT; ++i)
+                v[y][i] = y0 + y < parts
+                              ? __ldcg(reinterpret_cast<const float4*>(p.partial) + ((size_t)(y0 + y) * p.T + tile) * kF4 + i * 32 + lane)
+                              : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+            for (int y = 0; y < 2; ++y)
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                  const float4 a = v[y][mt * NT + nt];
+                  acc[mt][nt][0] += a.x, acc[mt][nt][1] += a.y, acc[mt][nt][2] += a.z, acc[mt][nt][3] += a.w;
+                }
+          }
+        }
+      }
+      // the epilogue transposes through the ring slot the warp has just multiplied, one sub-tile at a time
+      if (finish) {
+        float* sE = reinterpret_cast<float*>(ring + (cslot == 0 ? STAGES - 1 : cslot - 1) * kRoundStage);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+          if (tile * MT + mt < p.Tsub) tile_epilogue<NT>(p, acc[mt], tile * MT + mt, sE, lane, best, bidx);
+      }
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[mt][nt][c] = 0.0f;
+    if (kw > 1) __syncthreads();  // the partners' slots are read before anyone requests a stage into them
+  }
+  cp_async_wait<0>();
+
+  if (p.epilogue == EPI_F32 && p.argmax_partial && (lane & 1) == 0) {
+    const int req = lane >> 1;
+    if (req < NP && req < p.n)
+      p.argmax_partial[((size_t)(blockIdx.y * gridDim.x + blockIdx.x) * kRoundWarps + warp) * 16 + req] =
+          make_float2(best, __int_as_float(bidx));
+  }
+}
+
+struct RoundPlan {
+  int nt, stages, Q, S, parts, T, Tsub, ctas, kw;
+  size_t smem, partial_bytes;
+};
+
+RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
+  RoundPlan t;
+  t.nt = n <= 8 ? 1 : 2;
+  t.stages = t.nt == 1 ? 5 : 4;
+  const int quads = K / 256;
+  t.Q = 1;
+  for (int c = kMaxQuadsPerSlice; c >= 1; --c)
+    if (quads % c == 0) {
+      t.Q = c;
+      break;
+    }
+  const int slices = quads / t.Q;
+  // A CTA re-reads the activations of its part of K for every round, so K is cut into parts of at most four
+  // slices: beyond that the activations would outweigh the CTA's weights.
+  t.parts = 1;
+  while (slices % t.parts || slices / t.parts > 4) ++t.parts;
+  t.S = slices / t.parts;
+  t.Tsub = epilogue == EPI_SILU_PACK ? (N / 2 + 7) / 8 : (N + 15) / 16;
+  t.T = (t.Tsub + kRoundMT - 1) / kRoundMT;
+  int ctas = sm_count / t.parts;
+  if (ctas < 1) ctas = 1;
+  t.ctas = t.T < ctas ? t.T : ctas;
+  const int per_cta = (t.T + t.ctas - 1) / t.ctas;
+  int kw = 1;
+  while (kw * 2 <= kRoundWarps / per_cta && kw * 2 <= t.S * t.Q) kw *= 2;  // fill the CTA's warps, a stage each at least
+  t.kw = kw;
+  const int np = 8 * t.nt;
+  t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * (size_t)np * (t.Q * 512 + 16) + 2 * (size_t)t.Q * 4 * 16 * 4;
+  t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
+  return t;
+}
+
 template <int MT, int NT, int STAGES>
 size_t smem_bytes(int ks) {
   return (size_t)kWarps * STAGES * (16 * MT) * (kRowStride + kSbBytes) + (size_t)(8 * NT) * (ks * 2 + 16) +
@@ -450,23 +940,15 @@ __global__ void __launch_bounds__(256) argmax_finish_kernel(const float2* partia
 
 size_t gemm_partial_bytes(int N, int K, int epilogue) {
   const int sms = sm_count_or_default();
-  size_t need = 0;
-  for (int n = 8; n <= 16; n += 8) {  // the tilings: up to 8 requests, 9..16 requests (either CTA size)
-    for (int force = 1; force <= 2; ++force) {
-      const int saved = g_force_cfg;
-      g_force_cfg = n > 8 ? force : saved;
-      const size_t b = tiling_partial_bytes(choose_tiling(N, K, n, epilogue, sms));
-      g_force_cfg = saved;
-      if (b > need) need = b;
-    }
-  }
-  return need;
+  const size_t a = plan_rounds(N, K, 8, epilogue, sms).partial_bytes, b = plan_rounds(N, K, 16, epilogue, sms).partial_bytes;
+  return a > b ? a : b;
 }
 
-int gemm_counters_needed(int N) { return (N + 63) / 64 + 1; }
+int gemm_counters_needed(int N) { return (N + 15) / 16 + 1; }
 
 int gemm_row_blocks(int N, int K, int n, int epilogue) {
-  return choose_tiling(N, K, n, epilogue, sm_count_or_default()).rowblocks;
+  const RoundPlan t = plan_rounds(N, K, n, epilogue, sm_count_or_default());
+  return t.ctas * t.parts * kRoundWarps;  // one argmax partial per warp of the grid
 }
 
 cudaError_t gemm_init() {
@@ -483,6 +965,10 @@ cudaError_t gemm_init() {
     e = cudaFuncSetAttribute(q4_gemm_kernel<2, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_round_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_round_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   g_sm_count = sms;
@@ -496,9 +982,25 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
   }
   if (a.n <= 0) return cudaSuccess;
   if (a.N <= 0 || a.K <= 0 || (a.K % 256) || a.n > kMaxBatch) return cudaErrorInvalidValue;
-  if (a.epilogue == EPI_SILU_PACK && ((a.N % 16) || !a.out_xp || !a.out_xs)) return cudaErrorInvalidValue;
   const bool grouped = a.expert_ids != nullptr;
+  if (a.epilogue == EPI_SILU_PACK && ((a.N % 16) || !a.out_xp || (grouped && !a.out_xs))) return cudaErrorInvalidValue;
   if (grouped && (a.K > 2048 || !a.n_touched || a.max_slots < 1)) return cudaErrorInvalidValue;
+  if (!grouped) {
+    const RoundPlan t = plan_rounds(a.N, a.K, a.n, a.epilogue, g_sm_count);
+    RoundParams p;
+    p.qw = a.qw, p.scales = a.scales, p.biases = a.biases, p.xp = a.xp, p.xs = a.xs, p.out = a.out;
+    p.out_xp = a.out_xp, p.argmax_partial = a.argmax_partial, p.status = a.status;
+    p.N = a.N, p.K = a.K, p.n = a.n, p.out_stride = a.out_stride, p.epilogue = a.epilogue;
+    p.T = t.T, p.Tsub = t.Tsub, p.Q = t.Q, p.S = t.S, p.kw = t.kw;
+    p.partial = a.partial, p.counters = a.counters;
+    if (t.parts > 1 && (!a.partial || !a.counters || t.partial_bytes > a.partial_bytes || t.T > a.counters_len))
+      return cudaErrorInvalidValue;
+    const int elem = a.epilogue == EPI_F32 ? 4 : 2;
+    p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
+    const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
+    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
+    return launch_kernel(q4_round_kernel<2, 4>, grid, block, t.smem, s, p);
+  }
   const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;
   p.expert_ids = a.expert_ids, p.n_touched = a.n_touched, p.expert_rows = a.N;
