@@ -347,7 +347,7 @@ def main():
         top = max((k for k in kernels if k in class_bytes), key=lambda k: kernels[k]["share"])
         top_ms, top_cnt = prof[top]
         gbs = class_bytes[top] / (top_ms / top_cnt * 1e-3) / 1e9
-        roofline = {"kernel": class_kernel.get(top, "q4_gemm_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
+        roofline = {"kernel": class_kernel.get(top, "q4_round_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
                     "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": peak_kind,
                     "traffic": class_bytes[top] * traffic_ratio[top] if top in traffic_ratio else None,
                     "bytes_per_launch": float(class_bytes[top]), "us_per_launch": top_ms / top_cnt * 1e3,

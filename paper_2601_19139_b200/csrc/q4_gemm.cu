@@ -509,7 +509,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
-template <int NT, int STAGES>
+// ALL: the CTA has a single round and every slice of its part of K fits in shared memory at once (short
+// projections): all activations are requested up front and the warps run through their stages without the
+// per-slice barriers, whose cost and the exposed latency of each slice's copy would otherwise dominate.
+template <int NT, int STAGES, bool ALL>
 __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundParams p) {
   constexpr int NP = 8 * NT, MT = kRoundMT, RW = kRoundRows;
   constexpr int kEs = NP + 1;
@@ -529,8 +532,9 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   const int sum_bytes = Q * 4 * 16 * 4;    // group sums of a slice: [group][16]
 
   unsigned char* ring = smem + warp * (STAGES * kRoundStage);
-  unsigned char* sAct = smem + kRoundWarps * STAGES * kRoundStage;  // two buffers
-  float* sSum = reinterpret_cast<float*>(sAct + 2 * act_bytes);     // two buffers
+  const int nbuf = ALL ? S : 2;
+  unsigned char* sAct = smem + kRoundWarps * STAGES * kRoundStage;   // nbuf buffers
+  float* sSum = reinterpret_cast<float*>(sAct + nbuf * act_bytes);  // nbuf buffers
   (void)kEs;
 
   // the CTA's tiles and rounds
@@ -573,8 +577,10 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   int islot = 0, cslot = 0;
   const bool any = my_rounds > 0 && kp < SQ;
   // Weights do not depend on the preceding kernel: start streaming them before waiting for it.
+  // (With all slices resident a warp's last stage has no successor, so the slot it multiplied last stays free for
+  // the epilogue even if every slot is filled up front and refilled right after use: one more stage in flight.)
 #pragma unroll
-  for (int s = 0; s < STAGES - 1; ++s) {
+  for (int s = 0; s < (ALL ? STAGES : STAGES - 1); ++s) {
     if (any && ir < my_rounds) {
       issue_stage(islot, tile_of(ir), ij);
       ij += kw;
@@ -594,20 +600,30 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   grid_dependency_wait();
 
   // One bulk copy per request row of the slice (and one for its group sums), tracked by the buffer's mbarrier.
+  const uint32_t slice_bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
+  auto copy_slice = [&](int buf, int sl, uint64_t* bar) {
+    const int slice = blockIdx.y * S + sl;
+    for (int r = 0; r < NP; ++r)
+      bulk_copy_g2s(sAct + buf * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2), bar);
+    if (p.xs) bulk_copy_g2s(sSum + buf * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, bar);
+  };
   auto stage_acts = [&](int gstep) {
     if (threadIdx.x == 0) {
-      const int b = gstep & 1, slice = blockIdx.y * S + gstep % S;
-      const uint32_t bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
-      mbar_expect_tx(&s_mbar[b], bytes);
-      for (int r = 0; r < NP; ++r)
-        bulk_copy_g2s(sAct + b * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
-                      &s_mbar[b]);
-      if (p.xs) bulk_copy_g2s(sSum + b * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar[b]);
+      mbar_expect_tx(&s_mbar[gstep & 1], slice_bytes);
+      copy_slice(gstep & 1, gstep % S, &s_mbar[gstep & 1]);
     }
     __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
   };
   const int steps = R * S;
-  if (steps > 0) stage_acts(0);
+  if (ALL) {
+    if (threadIdx.x == 0 && steps > 0) {
+      mbar_expect_tx(&s_mbar[0], slice_bytes * (uint32_t)S);
+      for (int sl = 0; sl < S; ++sl) copy_slice(sl, sl, &s_mbar[0]);
+    }
+    __syncwarp();
+  } else if (steps > 0) {
+    stage_acts(0);
+  }
 
   float acc[MT][NT][4];
 #pragma unroll
@@ -623,34 +639,41 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   for (int r = 0; r < R; ++r) {
     for (int s = 0; s < S; ++s, ++gstep) {
       // the other buffer was last read in step gstep - 1, which every warp has left (barrier below)
-      if (gstep + 1 < steps) stage_acts(gstep + 1);
-      const int b = gstep & 1;
-      if (!mbar_wait(&s_mbar[b], (uint32_t)((gstep >> 1) & 1))) {
-        if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copy never landed: report, results are void
+      if (!ALL && gstep + 1 < steps) stage_acts(gstep + 1);
+      const int b = ALL ? s : (gstep & 1);
+      if (!ALL || s == 0) {
+        if (!mbar_wait(&s_mbar[ALL ? 0 : b], ALL ? 0u : (uint32_t)((gstep >> 1) & 1))) {
+          if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copy never landed: report, results are void
+        }
       }
       const unsigned char* sB = sAct + b * act_bytes;
       float* sX = sSum + b * (sum_bytes / 4);
-      if (!p.xs) {
-        // the producer left no group sums: add up the 64 staged elements of every (group, request)
-        for (int c = threadIdx.x; c < Q * 4 * NP; c += kRoundThreads) {
-          const int gq = c / NP, rq = c - gq * NP;
-          const uint4* src = reinterpret_cast<const uint4*>(sB + rq * b_stride + gq * 128);
+      if (!p.xs && (!ALL || s == 0)) {
+        // the producer left no group sums: add up the 64 staged elements of every (group, request) of the slice
+        // (of all slices when they are all resident)
+        const int per = Q * 4 * NP;
+        for (int c = threadIdx.x; c < (ALL ? S : 1) * per; c += kRoundThreads) {
+          const int sl = c / per, cc = c - sl * per;
+          const int gq = cc / NP, rq = cc - gq * NP;
+          const uint4* src = reinterpret_cast<const uint4*>(sAct + (b + sl) * act_bytes + rq * b_stride + gq * 128);
           float sum = 0.0f;
 #pragma unroll
           for (int i = 0; i < 8; ++i) sum += chunk_sum(src[i]);
-          sX[gq * 16 + rq] = sum;
+          sSum[(b + sl) * (sum_bytes / 4) + gq * 16 + rq] = sum;
         }
         __syncthreads();
       }
 
       while (any && cr == r && cr < my_rounds && cj < (s + 1) * Q) {
-        if (ir < my_rounds) {
-          issue_stage(islot, tile_of(ir), ij);
-          ij += kw;
-          if (ij >= SQ) ij = kp, ++ir;
-          if (++islot == STAGES) islot = 0;
+        if (!ALL) {
+          if (ir < my_rounds) {
+            issue_stage(islot, tile_of(ir), ij);
+            ij += kw;
+            if (ij >= SQ) ij = kp, ++ir;
+            if (++islot == STAGES) islot = 0;
+          }
+          cp_async_commit();
         }
-        cp_async_commit();
         cp_async_wait<STAGES - 1>();
         __syncwarp();
         const unsigned char* stg = ring + cslot * kRoundStage;
@@ -707,6 +730,15 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
           }
         }
         __syncwarp();
+        if (ALL) {  // refill the slot just multiplied
+          if (ir < my_rounds) {
+            issue_stage(islot, tile_of(ir), ij);
+            ij += kw;
+            if (ij >= SQ) ij = kp, ++ir;
+            if (++islot == STAGES) islot = 0;
+          }
+          cp_async_commit();
+        }
         cj += kw;
         if (cj >= SQ) cj = kp, ++cr;
       }
@@ -721,7 +753,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
           for (int nt = 0; nt < NT; ++nt)
             dst[(mt * NT + nt) * 32 + lane] = make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
       }
-      __syncthreads();
+      if (!ALL || (s == S - 1 && kw > 1)) __syncthreads();
     }
     // round end: the first warp of every tile adds its partners in warp order and applies the epilogue
     if (r < my_rounds && kp == 0) {
@@ -812,6 +844,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
 
 struct RoundPlan {
   int nt, stages, Q, S, parts, T, Tsub, ctas, kw;
+  bool all;  // every slice of the part resident at once (single round, few stages per warp)
   size_t smem, partial_bytes;
 };
 
@@ -842,7 +875,11 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   while (kw * 2 <= kRoundWarps / per_cta && kw * 2 <= t.S * t.Q) kw *= 2;  // fill the CTA's warps, a stage each at least
   t.kw = kw;
   const int np = 8 * t.nt;
-  t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * (size_t)np * (t.Q * 512 + 16) + 2 * (size_t)t.Q * 4 * 16 * 4;
+  // short projections: one round, at most four stages per warp -> all slices resident, two ring slots per warp
+  t.all = per_cta * kw <= kRoundWarps && t.S * t.Q <= 4 * kw;
+  if (t.all) t.stages = 2;
+  const int nbuf = t.all ? t.S : 2;
+  t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + nbuf * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
   return t;
 }
@@ -966,9 +1003,13 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<1, 5, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<2, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_round_kernel<1, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(q4_round_kernel<2, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   g_sm_count = sms;
@@ -998,8 +1039,12 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     const int elem = a.epilogue == EPI_F32 ? 4 : 2;
     p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
     const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
-    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
-    return launch_kernel(q4_round_kernel<2, 4>, grid, block, t.smem, s, p);
+    if (t.all) {
+      if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 2, true>, grid, block, t.smem, s, p);
+      return launch_kernel(q4_round_kernel<2, 2, true>, grid, block, t.smem, s, p);
+    }
+    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5, false>, grid, block, t.smem, s, p);
+    return launch_kernel(q4_round_kernel<2, 4, false>, grid, block, t.smem, s, p);
   }
   const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;
