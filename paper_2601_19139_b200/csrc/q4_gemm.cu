@@ -10,10 +10,14 @@
 // no dequantised weight is ever rounded to bf16; scale and bias (less 16 * scale,
 // which removes the offset again) are applied to the fp32 group sums.
 //
-// Layout of the work: see q4_round_kernel below (one CTA per SM walks its row tiles in rounds, whole K or a part
-// of it inside the CTA; the weight stream does not depend on the preceding kernel, so it is started before the
-// grid dependency is awaited).  q4_gemm_kernel is the older CTA-granular form (a CTA owns 128 rows and one
-// K-slice, split-K through global scratch); the grouped mode of the mixture-of-experts layers still runs on it.
+// Layout of the work.  One CTA of 16 warps per SM owns a contiguous range of 16-row tiles (and, for K > 4096, one
+// part of K).  q4_span_kernel serves CTAs with at most 16 tiles (the projections of a layer): every slice of the
+// operand is resident, each warp streams an equal contiguous span of the CTA's stages, partial tiles meet in shared
+// memory.  q4_round_kernel serves longer tile ranges (the LM head): rounds of 16 tiles, the operand slices double
+// buffered with a CTA barrier per slice.  In both the weight stream does not depend on the preceding kernel, so it
+// is started before the grid dependency is awaited.  q4_gemm_kernel is the older CTA-granular form (a CTA owns 128
+// rows and one K-slice, split-K through global scratch); the grouped mode of the mixture-of-experts layers still
+// runs on it.
 #include <stdlib.h>
 
 #include "common.cuh"
@@ -509,10 +513,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
-// ALL: the CTA has a single round and every slice of its part of K fits in shared memory at once (short
-// projections): all activations are requested up front and the warps run through their stages without the
-// per-slice barriers, whose cost and the exposed latency of each slice's copy would otherwise dominate.
-template <int NT, int STAGES, bool ALL>
+template <int NT, int STAGES>
 __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundParams p) {
   constexpr int NP = 8 * NT, MT = kRoundMT, RW = kRoundRows;
   constexpr int kEs = NP + 1;
@@ -532,9 +533,8 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   const int sum_bytes = Q * 4 * 16 * 4;    // group sums of a slice: [group][16]
 
   unsigned char* ring = smem + warp * (STAGES * kRoundStage);
-  const int nbuf = ALL ? S : 2;
-  unsigned char* sAct = smem + kRoundWarps * STAGES * kRoundStage;   // nbuf buffers
-  float* sSum = reinterpret_cast<float*>(sAct + nbuf * act_bytes);  // nbuf buffers
+  unsigned char* sAct = smem + kRoundWarps * STAGES * kRoundStage;  // two buffers
+  float* sSum = reinterpret_cast<float*>(sAct + 2 * act_bytes);     // two buffers
   (void)kEs;
 
   // the CTA's tiles and rounds
@@ -577,10 +577,8 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   int islot = 0, cslot = 0;
   const bool any = my_rounds > 0 && kp < SQ;
   // Weights do not depend on the preceding kernel: start streaming them before waiting for it.
-  // (With all slices resident a warp's last stage has no successor, so the slot it multiplied last stays free for
-  // the epilogue even if every slot is filled up front and refilled right after use: one more stage in flight.)
 #pragma unroll
-  for (int s = 0; s < (ALL ? STAGES : STAGES - 1); ++s) {
+  for (int s = 0; s < STAGES - 1; ++s) {
     if (any && ir < my_rounds) {
       issue_stage(islot, tile_of(ir), ij);
       ij += kw;
@@ -615,15 +613,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
     __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
   };
   const int steps = R * S;
-  if (ALL) {
-    if (threadIdx.x == 0 && steps > 0) {
-      mbar_expect_tx(&s_mbar[0], slice_bytes * (uint32_t)S);
-      for (int sl = 0; sl < S; ++sl) copy_slice(sl, sl, &s_mbar[0]);
-    }
-    __syncwarp();
-  } else if (steps > 0) {
-    stage_acts(0);
-  }
+  if (steps > 0) stage_acts(0);
 
   float acc[MT][NT][4];
 #pragma unroll
@@ -639,41 +629,34 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   for (int r = 0; r < R; ++r) {
     for (int s = 0; s < S; ++s, ++gstep) {
       // the other buffer was last read in step gstep - 1, which every warp has left (barrier below)
-      if (!ALL && gstep + 1 < steps) stage_acts(gstep + 1);
-      const int b = ALL ? s : (gstep & 1);
-      if (!ALL || s == 0) {
-        if (!mbar_wait(&s_mbar[ALL ? 0 : b], ALL ? 0u : (uint32_t)((gstep >> 1) & 1))) {
-          if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copy never landed: report, results are void
-        }
+      if (gstep + 1 < steps) stage_acts(gstep + 1);
+      const int b = gstep & 1;
+      if (!mbar_wait(&s_mbar[b], (uint32_t)((gstep >> 1) & 1))) {
+        if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copy never landed: report, results are void
       }
       const unsigned char* sB = sAct + b * act_bytes;
       float* sX = sSum + b * (sum_bytes / 4);
-      if (!p.xs && (!ALL || s == 0)) {
+      if (!p.xs) {
         // the producer left no group sums: add up the 64 staged elements of every (group, request) of the slice
-        // (of all slices when they are all resident)
-        const int per = Q * 4 * NP;
-        for (int c = threadIdx.x; c < (ALL ? S : 1) * per; c += kRoundThreads) {
-          const int sl = c / per, cc = c - sl * per;
-          const int gq = cc / NP, rq = cc - gq * NP;
-          const uint4* src = reinterpret_cast<const uint4*>(sAct + (b + sl) * act_bytes + rq * b_stride + gq * 128);
+        for (int c = threadIdx.x; c < Q * 4 * NP; c += kRoundThreads) {
+          const int gq = c / NP, rq = c - gq * NP;
+          const uint4* src = reinterpret_cast<const uint4*>(sB + rq * b_stride + gq * 128);
           float sum = 0.0f;
 #pragma unroll
           for (int i = 0; i < 8; ++i) sum += chunk_sum(src[i]);
-          sSum[(b + sl) * (sum_bytes / 4) + gq * 16 + rq] = sum;
+          sX[gq * 16 + rq] = sum;
         }
         __syncthreads();
       }
 
       while (any && cr == r && cr < my_rounds && cj < (s + 1) * Q) {
-        if (!ALL) {
-          if (ir < my_rounds) {
-            issue_stage(islot, tile_of(ir), ij);
-            ij += kw;
-            if (ij >= SQ) ij = kp, ++ir;
-            if (++islot == STAGES) islot = 0;
-          }
-          cp_async_commit();
+        if (ir < my_rounds) {
+          issue_stage(islot, tile_of(ir), ij);
+          ij += kw;
+          if (ij >= SQ) ij = kp, ++ir;
+          if (++islot == STAGES) islot = 0;
         }
+        cp_async_commit();
         cp_async_wait<STAGES - 1>();
         __syncwarp();
         const unsigned char* stg = ring + cslot * kRoundStage;
@@ -730,15 +713,6 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
           }
         }
         __syncwarp();
-        if (ALL) {  // refill the slot just multiplied
-          if (ir < my_rounds) {
-            issue_stage(islot, tile_of(ir), ij);
-            ij += kw;
-            if (ij >= SQ) ij = kp, ++ir;
-            if (++islot == STAGES) islot = 0;
-          }
-          cp_async_commit();
-        }
         cj += kw;
         if (cj >= SQ) cj = kp, ++cr;
       }
@@ -753,7 +727,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
           for (int nt = 0; nt < NT; ++nt)
             dst[(mt * NT + nt) * 32 + lane] = make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
       }
-      if (!ALL || (s == S - 1 && kw > 1)) __syncthreads();
+      __syncthreads();
     }
     // round end: the first warp of every tile adds its partners in warp order and applies the epilogue
     if (r < my_rounds && kp == 0) {
@@ -842,9 +816,294 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   }
 }
 
+// ---- span kernel: projections whose CTAs hold at most 16 row tiles ------------------------------------------------
+// All K-slices of the CTA's part of K (at most four) are resident in shared memory, so nothing ties the warps to one
+// another while they multiply.  The CTA's stages, row tile major, are cut into 16 equal contiguous spans, one per
+// warp: every warp streams the same number of stages (to within one) whatever the number of tiles, a span covers the
+// tail of one tile and the head of the next at most, and each warp refills the ring slot it has just multiplied.
+// At the end the warps leave their (one or two) partial sums in shared memory, and the warp that holds a tile's first
+// stage adds the tile's partial sums in warp order and applies the epilogue.
+__device__ __forceinline__ void span_issue_stage(const RoundParams& p, unsigned char* stg, int sub, int stage_k, bool silu,
+                                                 int half_n, int lane) {
+  auto row_of = [&](int r) -> int {
+    if (!silu) return min(sub * 16 + r, p.N - 1);
+    return r < 8 ? min(sub * 8 + r, half_n - 1) : min(half_n + sub * 8 + (r - 8), p.N - 1);
+  };
+  const int kq = stage_k * 256;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 4 + (lane >> 3);
+    const unsigned char* src =
+        reinterpret_cast<const unsigned char*>(p.qw + (size_t)row_of(r) * (p.K >> 3) + (kq >> 3)) + (lane & 7) * 16;
+    cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), src);
+  }
+  if (lane < 16) {
+    const size_t off = (size_t)row_of(lane) * (p.K >> 6) + (kq >> 6);
+    cp_async8(stg + 16 * 128 + lane * kSbBytes, p.scales + off);
+    cp_async8(stg + 16 * 128 + lane * kSbBytes + 8, p.biases + off);
+  }
+}
+
+// acc += the stage's 16 rows x 256 input features against the staged operand (sB: the slice, sX: its group sums,
+// cq: the stage's place in the slice).
+template <int NT>
+__device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, const unsigned char* sB, const float* sX,
+                                                    int b_stride, int cq, int g, int t, float (&acc)[NT][4]) {
+  uint2 sc[2], bi[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const uint4 v = *reinterpret_cast<const uint4*>(stg + 16 * 128 + (g + 8 * h) * kSbBytes);
+    sc[h] = make_uint2(v.x, v.y);
+    bi[h] = make_uint2(v.z, v.w);
+  }
+#pragma unroll
+  for (int gi = 0; gi < 4; ++gi) {
+    const int gidx = cq * 4 + gi;
+    uint4 bf[NT][2];
+    float2 xs[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const unsigned char* bp = sB + (nt * 8 + g) * b_stride + gidx * 128 + t * 32;
+      bf[nt][0] = *reinterpret_cast<const uint4*>(bp);
+      bf[nt][1] = *reinterpret_cast<const uint4*>(bp + 16);
+      xs[nt] = *reinterpret_cast<const float2*>(sX + gidx * 16 + nt * 8 + 2 * t);
+    }
+    // 16-byte chunk c of row r sits at chunk c ^ (r & 7); rows g and g + 8 share the swizzle
+    const int woff = g * 128 + (((gi * 2 + (t >> 1)) ^ g) << 4) + (t & 1) * 8;
+    const uint2 wl = *reinterpret_cast<const uint2*>(stg + woff);
+    const uint2 wh = *reinterpret_cast<const uint2*>(stg + woff + 8 * 128);
+    uint32_t l0[4], l1[4], h0[4], h1[4];
+    unpack_word(wl.x, l0);
+    unpack_word(wl.y, l1);
+    unpack_word(wh.x, h0);
+    unpack_word(wh.y, h1);
+    // sum (16 + q) x = 16 X + sum q x, so the bias that multiplies X becomes b - 16 s
+    const float s_lo = bf16_at(sc[0], gi), s_hi = bf16_at(sc[1], gi);
+    const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[1], gi));
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      float pc[4];
+      mma_bf16_first(pc, l0[0], h0[0], l0[1], h0[1], bf[nt][0].x, bf[nt][0].y);
+      mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
+      mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
+      mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
+      acc[nt][0] = fmaf(s_lo, pc[0], fmaf(b_lo, xs[nt].x, acc[nt][0]));
+      acc[nt][1] = fmaf(s_lo, pc[1], fmaf(b_lo, xs[nt].y, acc[nt][1]));
+      acc[nt][2] = fmaf(s_hi, pc[2], fmaf(b_hi, xs[nt].x, acc[nt][2]));
+      acc[nt][3] = fmaf(s_hi, pc[3], fmaf(b_hi, xs[nt].y, acc[nt][3]));
+    }
+  }
+}
+
+template <int NT, int STAGES>
+__global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundParams p) {
+  static_assert(kRoundMT == 1, "the span kernel works on 16-row tiles");
+  constexpr int NP = 8 * NT, W = kRoundWarps;
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) uint64_t s_mbar;
+
+  grid_launch_dependents();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const bool silu = p.epilogue == EPI_SILU_PACK;
+  const int half_n = p.N >> 1;
+  const int Q = p.Q, S = p.S, SQ = S * Q;
+  const int parts = gridDim.y, part_j0 = blockIdx.y * SQ;
+  const int ks = Q * 256;
+  const int b_stride = ks * 2 + 16;
+  const int act_bytes = NP * b_stride;
+  const int sum_bytes = Q * 4 * 16 * 4;
+
+  unsigned char* ring = smem + warp * (STAGES * kRoundStage);
+  unsigned char* sAct = smem + W * STAGES * kRoundStage;             // S buffers; the partial sums at the end
+  float* sSum = reinterpret_cast<float*>(sAct + S * act_bytes);     // S buffers
+
+  // the CTA's tiles, and this warp's span of their stages
+  const int t0 = (int)((long long)blockIdx.x * p.T / gridDim.x), t1 = (int)((long long)(blockIdx.x + 1) * p.T / gridDim.x);
+  const int Tc = t1 - t0, Lc = Tc * SQ;
+  auto span_begin = [&](int w) -> int { return w * Lc / W; };
+  const int a = span_begin(warp), cnt = span_begin(warp + 1) - a;
+  const int tlA = a / SQ, jA0 = a - tlA * SQ;
+  const int lenA = min(cnt, SQ - jA0);  // stages in the first tile; the rest belong to tile tlA + 1, from its stage 0
+  auto stage_of = [&](int i, int& tl, int& j) {
+    if (i < lenA) tl = tlA, j = jA0 + i;
+    else tl = tlA + 1, j = i - lenA;
+  };
+
+  // Weights do not depend on the preceding kernel: fill the ring before waiting for it.
+#pragma unroll
+  for (int i = 0; i < STAGES; ++i) {
+    if (i < cnt) {
+      int tl, j;
+      stage_of(i, tl, j);
+      span_issue_stage(p, ring + i * kRoundStage, t0 + tl, part_j0 + j, silu, half_n, lane);
+    }
+    cp_async_commit();
+  }
+
+  if (threadIdx.x == 0) {
+    mbar_init(&s_mbar, 1u);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  grid_dependency_wait();
+
+  // every slice of the operand (and its group sums): one bulk copy per request row, all on one mbarrier
+  if (threadIdx.x == 0) {
+    const uint32_t slice_bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
+    mbar_expect_tx(&s_mbar, slice_bytes * (uint32_t)S);
+    for (int sl = 0; sl < S; ++sl) {
+      const int slice = blockIdx.y * S + sl;
+      for (int r = 0; r < NP; ++r)
+        bulk_copy_g2s(sAct + sl * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
+                      &s_mbar);
+      if (p.xs) bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
+    }
+  }
+  __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
+  if (!mbar_wait(&s_mbar, 0u)) {
+    if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copies never landed: report, results are void
+  }
+  if (!p.xs) {
+    // the producer left no group sums: add up the 64 staged elements of every (slice, group, request)
+    const int per = Q * 4 * NP;
+    for (int c = threadIdx.x; c < S * per; c += kRoundThreads) {
+      const int sl = c / per, cc = c - sl * per;
+      const int gq = cc / NP, rq = cc - gq * NP;
+      const uint4* src = reinterpret_cast<const uint4*>(sAct + sl * act_bytes + rq * b_stride + gq * 128);
+      float sum = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sum += chunk_sum(src[i]);
+      sSum[sl * (sum_bytes / 4) + gq * 16 + rq] = sum;
+    }
+    __syncthreads();
+  }
+
+  float acc[NT][4], first[NT][4];  // the tile being multiplied; the finished part of the span's first tile
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f, first[nt][c] = 0.0f;
+
+  int slot = 0;
+  for (int i = 0; i < cnt; ++i) {
+    cp_async_wait<STAGES - 1>();
+    __syncwarp();
+    int tl, j;
+    stage_of(i, tl, j);
+    if (i == lenA) {  // the span moves on to its second tile
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) first[nt][c] = acc[nt][c], acc[nt][c] = 0.0f;
+    }
+    const int sl = j / Q, cq = j - sl * Q;
+    span_multiply_stage<NT>(ring + slot * kRoundStage, sAct + sl * act_bytes, sSum + sl * (sum_bytes / 4), b_stride, cq, g, t,
+                            acc);
+    __syncwarp();
+    if (i + STAGES < cnt) {  // refill the slot just multiplied
+      int tl2, j2;
+      stage_of(i + STAGES, tl2, j2);
+      span_issue_stage(p, ring + slot * kRoundStage, t0 + tl2, part_j0 + j2, silu, half_n, lane);
+    }
+    cp_async_commit();
+    if (++slot == STAGES) slot = 0;
+  }
+  cp_async_wait<0>();
+  const bool two = cnt > lenA;  // the span reached a second tile: `first` holds tile tlA, acc tile tlA + 1
+  __syncthreads();              // nobody reads the operand any more: its buffers take the partial sums
+
+  // partial sums, lane-major: [warp][first or second tile of the span][NT][32 lanes] float4
+  float4* sP = reinterpret_cast<float4*>(sAct);
+  if (cnt > 0) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const float (&fa)[4] = two ? first[nt] : acc[nt];
+      sP[((warp * 2 + 0) * NT + nt) * 32 + lane] = make_float4(fa[0], fa[1], fa[2], fa[3]);
+      if (two) sP[((warp * 2 + 1) * NT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+    }
+  }
+  __syncthreads();
+
+  float best = -INFINITY;
+  int bidx = 0x7fffffff;
+  // The warp whose span holds a tile's first stage finishes the tile: its own first tile if the span starts at the
+  // tile's stage 0, and its second tile always.
+  for (int which = 0; which < 2; ++which) {
+    const bool own = which == 0 ? (cnt > 0 && jA0 == 0) : two;
+    if (!own) continue;
+    const int tl = tlA + which;
+    const int wlast = ((tl * SQ + SQ) * W - 1) / Lc;  // the warp whose span holds the tile's last stage
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+    for (int w2 = warp; w2 <= wlast; ++w2) {
+      if (span_begin(w2 + 1) == span_begin(w2)) continue;   // an empty span (fewer stages than warps)
+      const int sel = (span_begin(w2) / SQ == tl) ? 0 : 1;  // the tile is that span's first or second
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float4 v = sP[((w2 * 2 + sel) * NT + nt) * 32 + lane];
+        acc[nt][0] += v.x, acc[nt][1] += v.y, acc[nt][2] += v.z, acc[nt][3] += v.w;
+      }
+    }
+    const int tile = t0 + tl;
+    bool finish = true;
+    if (parts > 1) {
+      // several CTAs hold parts of this tile's sums: publish, and the last to arrive adds them in part order
+      float4* part = reinterpret_cast<float4*>(p.partial) + ((size_t)blockIdx.y * p.T + tile) * (32 * NT);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) part[nt * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+      __threadfence();
+      __syncwarp();
+      int prev = 0;
+      if (lane == 0) prev = atomicAdd(p.counters + tile, 1);
+      prev = __shfl_sync(0xffffffffu, prev, 0);
+      finish = prev == parts - 1;
+      if (finish) {
+        __threadfence();
+        if (lane == 0) p.counters[tile] = 0;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+        for (int y0 = 0; y0 < parts; y0 += 4) {  // four parts at a time: their loads go out together
+          float4 v[4][NT];
+#pragma unroll
+          for (int y = 0; y < 4; ++y)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+              v[y][nt] = y0 + y < parts ? __ldcg(reinterpret_cast<const float4*>(p.partial) +
+                                                 ((size_t)(y0 + y) * p.T + tile) * (32 * NT) + nt * 32 + lane)
+                                        : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+          for (int y = 0; y < 4; ++y)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+              acc[nt][0] += v[y][nt].x, acc[nt][1] += v[y][nt].y, acc[nt][2] += v[y][nt].z, acc[nt][3] += v[y][nt].w;
+        }
+      }
+    }
+    // the epilogue transposes through the warp's ring, which is idle now
+    if (finish && tile < p.Tsub) tile_epilogue<NT>(p, acc, tile, reinterpret_cast<float*>(ring), lane, best, bidx);
+  }
+
+  if (p.epilogue == EPI_F32 && p.argmax_partial && (lane & 1) == 0) {
+    const int req = lane >> 1;
+    if (req < NP && req < p.n)
+      p.argmax_partial[((size_t)(blockIdx.y * gridDim.x + blockIdx.x) * W + warp) * 16 + req] =
+          make_float2(best, __int_as_float(bidx));
+  }
+}
+
+int g_part_slices = 4;  // K-slices per part of K; debugging aid: Q4D_GEMM_PART_SLICES
+
 struct RoundPlan {
   int nt, stages, Q, S, parts, T, Tsub, ctas, kw;
-  bool all;  // every slice of the part resident at once (single round, few stages per warp)
+  bool span;  // at most 16 tiles per CTA: the span kernel
+  int span_stages;
+  size_t span_smem;
   size_t smem, partial_bytes;
 };
 
@@ -863,7 +1122,7 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   // A CTA re-reads the activations of its part of K for every round, so K is cut into parts of at most four
   // slices: beyond that the activations would outweigh the CTA's weights.
   t.parts = 1;
-  while (slices % t.parts || slices / t.parts > 4) ++t.parts;
+  while (slices % t.parts || slices / t.parts > g_part_slices) ++t.parts;
   t.S = slices / t.parts;
   t.Tsub = epilogue == EPI_SILU_PACK ? (N / 2 + 7) / 8 : (N + 15) / 16;
   t.T = (t.Tsub + kRoundMT - 1) / kRoundMT;
@@ -875,12 +1134,13 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   while (kw * 2 <= kRoundWarps / per_cta && kw * 2 <= t.S * t.Q) kw *= 2;  // fill the CTA's warps, a stage each at least
   t.kw = kw;
   const int np = 8 * t.nt;
-  // short projections: one round, at most four stages per warp -> all slices resident, two ring slots per warp
-  t.all = per_cta * kw <= kRoundWarps && t.S * t.Q <= 4 * kw;
-  if (t.all) t.stages = 2;
-  const int nbuf = t.all ? t.S : 2;
-  t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + nbuf * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
+  t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
+  t.span = per_cta <= kRoundWarps && kRoundMT == 1;
+  t.span_stages = t.nt == 1 ? 4 : (t.S <= 2 ? 4 : (t.S <= 3 ? 3 : 2));
+  const size_t operand = t.S * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
+  const size_t handover = (size_t)kRoundWarps * 2 * 16 * np * sizeof(float);  // two partial tiles per warp, in the operand's place
+  t.span_smem = (size_t)kRoundWarps * t.span_stages * kRoundStage + (operand > handover ? operand : handover);
   return t;
 }
 
@@ -1003,15 +1263,16 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<1, 5, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<2, 4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<1, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<2, 2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
+  if (const char* f = getenv("Q4D_GEMM_PART_SLICES")) g_part_slices = atoi(f) < 1 ? 1 : (atoi(f) > 4 ? 4 : atoi(f));
   g_sm_count = sms;
   return cudaSuccess;
 }
@@ -1039,12 +1300,14 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     const int elem = a.epilogue == EPI_F32 ? 4 : 2;
     p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
     const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
-    if (t.all) {
-      if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 2, true>, grid, block, t.smem, s, p);
-      return launch_kernel(q4_round_kernel<2, 2, true>, grid, block, t.smem, s, p);
+    if (t.span) {
+      if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 4>, grid, block, t.span_smem, s, p);
+      if (t.span_stages == 4) return launch_kernel(q4_span_kernel<2, 4>, grid, block, t.span_smem, s, p);
+      if (t.span_stages == 3) return launch_kernel(q4_span_kernel<2, 3>, grid, block, t.span_smem, s, p);
+      return launch_kernel(q4_span_kernel<2, 2>, grid, block, t.span_smem, s, p);
     }
-    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5, false>, grid, block, t.smem, s, p);
-    return launch_kernel(q4_round_kernel<2, 4, false>, grid, block, t.smem, s, p);
+    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
+    return launch_kernel(q4_round_kernel<2, 4>, grid, block, t.smem, s, p);
   }
   const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;

@@ -63,6 +63,8 @@ GEMM_CASES = [
     # N, K, n  -- several row blocks and K slices, ragged N, every batch size class
     (4096, 1024, 1), (4096, 1024, 16), (1024, 2048, 3), (1024, 3072, 16), (6144, 1024, 8), (6144, 4096, 9),
     (272, 256, 5), (5000, 512, 16), (4096, 12288, 2), (130, 768, 16),
+    # K in three parts at the full batch; many rounds per CTA with a ragged last tile; a single tile
+    (4096, 12288, 16), (40010, 512, 12), (16, 256, 16), (48, 1024, 4),
 ]
 
 
