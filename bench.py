@@ -334,7 +334,7 @@ def main():
             touched = shape.n_experts * (1.0 - (1.0 - shape.top_k / shape.n_experts) ** n)
             class_bytes["moe_gate_up"] = touched * shp.q4_bytes(2 * shape.expert_inter, H)
             class_bytes["moe_down"] = touched * shp.q4_bytes(H, shape.expert_inter)
-        class_kernel = {"attention": "paged_attention_kernel", "moe_gate_up": "q4_gemm_kernel", "moe_down": "q4_gemm_kernel"}
+        class_kernel = {"attention": "paged_attention_kernel", "lm_head": "q4_round_kernel", "moe_gate_up": "q4_gemm_kernel", "moe_down": "q4_gemm_kernel"}
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped
         # batch-16 case (see profiles/); traffic is proportional to the bytes streamed, so it is scaled to this launch.
         traffic_ratio = {"gemm_gate_up": 1.006, "attention": 1.005}
@@ -347,7 +347,7 @@ def main():
         top = max((k for k in kernels if k in class_bytes), key=lambda k: kernels[k]["share"])
         top_ms, top_cnt = prof[top]
         gbs = class_bytes[top] / (top_ms / top_cnt * 1e-3) / 1e9
-        roofline = {"kernel": class_kernel.get(top, "q4_round_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
+        roofline = {"kernel": class_kernel.get(top, "q4_span_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
                     "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": peak_kind,
                     "traffic": class_bytes[top] * traffic_ratio[top] if top in traffic_ratio else None,
                     "bytes_per_launch": float(class_bytes[top]), "us_per_launch": top_ms / top_cnt * 1e3,

@@ -599,18 +599,17 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
 
   // One bulk copy per request row of the slice (and one for its group sums), tracked by the buffer's mbarrier.
   const uint32_t slice_bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
-  auto copy_slice = [&](int buf, int sl, uint64_t* bar) {
-    const int slice = blockIdx.y * S + sl;
-    for (int r = 0; r < NP; ++r)
-      bulk_copy_g2s(sAct + buf * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2), bar);
-    if (p.xs) bulk_copy_g2s(sSum + buf * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, bar);
-  };
-  auto stage_acts = [&](int gstep) {
-    if (threadIdx.x == 0) {
-      mbar_expect_tx(&s_mbar[gstep & 1], slice_bytes);
-      copy_slice(gstep & 1, gstep % S, &s_mbar[gstep & 1]);
+  auto stage_acts = [&](int gstep) {  // the lanes of warp 0 issue the copies side by side
+    if (warp == 0) {
+      const int buf = gstep & 1, slice = blockIdx.y * S + gstep % S;
+      if (lane == 0) mbar_expect_tx(&s_mbar[buf], slice_bytes);
+      if (lane < NP)
+        bulk_copy_g2s(sAct + buf * act_bytes + lane * b_stride, p.xp + (size_t)lane * p.K + (size_t)slice * ks,
+                      (uint32_t)(ks * 2), &s_mbar[buf]);
+      else if (lane == NP && p.xs)
+        bulk_copy_g2s(sSum + buf * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar[buf]);
     }
-    __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
+    __syncwarp();  // lanes that have nothing to issue go on to poll the mbarrier: they must not starve the others
   };
   const int steps = R * S;
   if (steps > 0) stage_acts(0);
@@ -949,19 +948,21 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
 
   grid_dependency_wait();
 
-  // every slice of the operand (and its group sums): one bulk copy per request row, all on one mbarrier
-  if (threadIdx.x == 0) {
-    const uint32_t slice_bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
-    mbar_expect_tx(&s_mbar, slice_bytes * (uint32_t)S);
-    for (int sl = 0; sl < S; ++sl) {
-      const int slice = blockIdx.y * S + sl;
-      for (int r = 0; r < NP; ++r)
+  // every slice of the operand (and its group sums): one bulk copy per request row, all on one mbarrier, issued by
+  // the lanes of warp 0 side by side (a single thread would spend microseconds issuing up to 68 copies)
+  if (warp == 0) {
+    if (lane == 0) mbar_expect_tx(&s_mbar, (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0)) * (uint32_t)S);
+    const int per = NP + 1;  // copies per slice: the rows, then the sums
+    for (int i = lane; i < S * per; i += 32) {
+      const int sl = i / per, r = i - sl * per, slice = blockIdx.y * S + sl;
+      if (r < NP)
         bulk_copy_g2s(sAct + sl * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
                       &s_mbar);
-      if (p.xs) bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
+      else if (p.xs)
+        bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
     }
   }
-  __syncwarp();  // the other lanes of the issuing warp go on to poll the mbarrier: they must not starve lane 0
+  __syncwarp();  // lanes that have nothing to issue go on to poll the mbarrier: they must not starve the others
   if (!mbar_wait(&s_mbar, 0u)) {
     if (lane == 0 && p.status) atomicExch(p.status, 3u);  // the copies never landed: report, results are void
   }
