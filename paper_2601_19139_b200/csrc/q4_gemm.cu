@@ -920,8 +920,11 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
   // the CTA's tiles, and this warp's span of their stages
   const int t0 = (int)((long long)blockIdx.x * p.T / gridDim.x), t1 = (int)((long long)(blockIdx.x + 1) * p.T / gridDim.x);
   const int Tc = t1 - t0, Lc = Tc * SQ;
-  auto span_begin = [&](int w) -> int { return w * Lc / W; };
-  const int a = span_begin(warp), cnt = span_begin(warp + 1) - a;
+  // Span i belongs to warp (i % 4) * 4 + i / 4: when only every second or fourth span holds a stage (few stages per
+  // CTA) the busy warps still spread over the four schedulers of the SM.
+  const int span = (warp & 3) * 4 + (warp >> 2);
+  auto span_begin = [&](int i) -> int { return i * Lc / W; };
+  const int a = span_begin(span), cnt = span_begin(span + 1) - a;
   const int tlA = a / SQ, jA0 = a - tlA * SQ;
   const int lenA = min(cnt, SQ - jA0);  // stages in the first tile; the rest belong to tile tlA + 1, from its stage 0
   auto stage_of = [&](int i, int& tl, int& j) {
@@ -1015,32 +1018,32 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
   const bool two = cnt > lenA;  // the span reached a second tile: `first` holds tile tlA, acc tile tlA + 1
   __syncthreads();              // nobody reads the operand any more: its buffers take the partial sums
 
-  // partial sums, lane-major: [warp][first or second tile of the span][NT][32 lanes] float4
+  // partial sums, lane-major: [span][first or second tile of the span][NT][32 lanes] float4
   float4* sP = reinterpret_cast<float4*>(sAct);
   if (cnt > 0) {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const float (&fa)[4] = two ? first[nt] : acc[nt];
-      sP[((warp * 2 + 0) * NT + nt) * 32 + lane] = make_float4(fa[0], fa[1], fa[2], fa[3]);
-      if (two) sP[((warp * 2 + 1) * NT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+      sP[((span * 2 + 0) * NT + nt) * 32 + lane] = make_float4(fa[0], fa[1], fa[2], fa[3]);
+      if (two) sP[((span * 2 + 1) * NT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
     }
   }
   __syncthreads();
 
   float best = -INFINITY;
   int bidx = 0x7fffffff;
-  // The warp whose span holds a tile's first stage finishes the tile: its own first tile if the span starts at the
+  // The warp whose span holds a tile's first stage finishes the tile (it adds the spans' partial sums in span order): its own first tile if the span starts at the
   // tile's stage 0, and its second tile always.
   for (int which = 0; which < 2; ++which) {
     const bool own = which == 0 ? (cnt > 0 && jA0 == 0) : two;
     if (!own) continue;
     const int tl = tlA + which;
-    const int wlast = ((tl * SQ + SQ) * W - 1) / Lc;  // the warp whose span holds the tile's last stage
+    const int last = ((tl * SQ + SQ) * W - 1) / Lc;  // the span that holds the tile's last stage
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
-    for (int w2 = warp; w2 <= wlast; ++w2) {
+    for (int w2 = span; w2 <= last; ++w2) {
       if (span_begin(w2 + 1) == span_begin(w2)) continue;   // an empty span (fewer stages than warps)
       const int sel = (span_begin(w2) / SQ == tl) ? 0 : 1;  // the tile is that span's first or second
 #pragma unroll
@@ -1138,7 +1141,10 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
   t.span = per_cta <= kRoundWarps && kRoundMT == 1;
-  t.span_stages = t.nt == 1 ? 4 : (t.S <= 2 ? 4 : (t.S <= 3 ? 3 : 2));
+  // two ring slots per warp (every slot is refilled as soon as it is multiplied); four for <= 8 requests and
+  // long K, where the operand is half the size and the multiply loop shorter.  Small footprints matter: the next
+  // projection's CTAs can then become resident, and request their weights, before this one has left the SM.
+  t.span_stages = (t.nt == 1 && t.S >= 3) ? 4 : 2;
   const size_t operand = t.S * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   const size_t handover = (size_t)kRoundWarps * 2 * 16 * np * sizeof(float);  // two partial tiles per warp, in the operand's place
   t.span_smem = (size_t)kRoundWarps * t.span_stages * kRoundStage + (operand > handover ? operand : handover);
@@ -1268,8 +1274,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_round_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
@@ -1302,9 +1307,8 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
     const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
     if (t.span) {
+      if (t.nt == 1 && t.span_stages == 2) return launch_kernel(q4_span_kernel<1, 2>, grid, block, t.span_smem, s, p);
       if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 4>, grid, block, t.span_smem, s, p);
-      if (t.span_stages == 4) return launch_kernel(q4_span_kernel<2, 4>, grid, block, t.span_smem, s, p);
-      if (t.span_stages == 3) return launch_kernel(q4_span_kernel<2, 3>, grid, block, t.span_smem, s, p);
       return launch_kernel(q4_span_kernel<2, 2>, grid, block, t.span_smem, s, p);
     }
     if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
