@@ -243,7 +243,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
  * memory-pool callback, or a serving loop where cudaMalloc is banned because it synchronises the
  * device.  Arguments and results are those of q4d_q4_gemm without `scratch`: the split-K scratch is
  * a fixed array inside the library (q4d_noalloc_max_scratch_bytes() = 8 MiB of partial sums, plus
- * 4096 row-block counters and 0.6 MiB in which the activations are rearranged for the kernel) that
+ * 4096 row-tile counters and 0.6 MiB in which the activations are rearranged for the kernel) that
  * every GPU holds from the moment the library is loaded until the process exits.  The call allocates
  * and frees nothing.
  *  - Projections whose split-K partial sums exceed the array, or with K > 16384, are refused with

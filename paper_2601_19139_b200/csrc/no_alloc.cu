@@ -19,7 +19,7 @@
 
 namespace {
 
-constexpr size_t kCounterBytes = 16 * 1024;          // 4096 row-block counters
+constexpr size_t kCounterBytes = 16 * 1024;          // 4096 row-tile counters
 constexpr size_t kPartialBytes = 8ull << 20;         // split-K partial sums
 constexpr int kMaxK = 16384;                         // widest input the operand buffers hold
 constexpr size_t kOperandBytes = (size_t)16 * kMaxK * 2 + (size_t)(kMaxK / 64) * 16 * 4;  // operand + group sums

@@ -218,6 +218,9 @@ def test_rope_append_matches_oracle(q4d, nq, nkv, qk_norm):
     (32, 4, [513, 129, 4000], 0),
     (8, 8, [50], 0),
     (32, 2, [333, 90], 128),
+    # more than eight chunks per request: eleven 12-tile chunks with a 3-tile tail, and nine planner-sized chunks
+    (32, 4, [1953, 194, 1036], 192),
+    (32, 8, [9000, 40], 0),
 ])
 def test_paged_attention_matches_oracle(q4d, nq, nkv, lens, chunk):
     n = len(lens)

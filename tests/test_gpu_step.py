@@ -238,6 +238,19 @@ def test_moe_30b_shape_layers_and_head_teacher_forced(q4d):
     assert emax <= LOGIT_TOL and same == n
 
 
+@pytest.mark.parametrize("nq,nkv,lens", [(16, 8, [9000, 200, 1500]), (32, 4, [9000, 100])])
+def test_long_request_many_chunks_layers_teacher_forced(q4d, nq, nkv, lens):
+    """One request far longer than the others: its KV is cut into dozens of chunks (29 with 8 kv heads, 71 with 4)
+    that the attention kernel prepares q for, appends to and merges itself; two layers of the 0.6B width, each from
+    the oracle's input."""
+    import dataclasses
+    shape = dataclasses.replace(shapes.QWEN3_0P6B, name=f"qwen3-0.6b-shaped-2layers-{nq}q{nkv}kv", n_layers=2,
+                                n_q_heads=nq, n_kv_heads=nkv)
+    sc = Scenario(shape, lens, seed=9)
+    _, emax, same, n = _layerwise(q4d, sc)
+    assert emax <= LOGIT_TOL and same == n
+
+
 def test_qwen3_0p6b_single_request_step(q4d):
     """Full 0.6B shape, batch 1, KV length 256, one whole step: bounded by the oracle's own fp32-accumulation drift."""
     sc = Scenario(shapes.QWEN3_0P6B, [256], seed=0)
