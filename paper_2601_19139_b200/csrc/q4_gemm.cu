@@ -479,10 +479,7 @@ struct RoundParams {
   int vec_ok;
 };
 
-#ifndef Q4D_ROUND_MT
-#define Q4D_ROUND_MT 1
-#endif
-constexpr int kRoundMT = Q4D_ROUND_MT;
+constexpr int kRoundMT = 1;  // sub-tiles of 16 rows per warp tile (2, with 8 warps of 198 registers, measured no faster)
 constexpr int kRoundWarps = 16 / kRoundMT, kRoundThreads = 32 * kRoundWarps;
 // a stage: 16 MT rows of 128 B of codes, 16-byte chunks swizzled by row, then the rows' scales and biases
 constexpr int kRoundRows = 16 * kRoundMT, kRoundStage = kRoundRows * (128 + kSbBytes);
