@@ -10,10 +10,10 @@
 // no dequantised weight is ever rounded to bf16; scale and bias (less 16 * scale,
 // which removes the offset again) are applied to the fp32 group sums.
 //
-// Layout of the work.  One CTA of 16 warps per SM owns a contiguous range of 16-row tiles (and, for K > 4096, one
-// part of K).  q4_span_kernel serves CTAs with at most 16 tiles (the projections of a layer): every slice of the
+// Layout of the work.  One CTA of 12 warps per SM owns a contiguous range of 16-row tiles (and, for K > 4096, one
+// part of K).  q4_span_kernel serves CTAs with at most 12 tiles (the projections of a layer): every slice of the
 // operand is resident, each warp streams an equal contiguous span of the CTA's stages, partial tiles meet in shared
-// memory.  q4_round_kernel serves longer tile ranges (the LM head): rounds of 16 tiles, the operand slices double
+// memory.  q4_round_kernel serves longer tile ranges (the LM head): rounds of 12 tiles, the operand slices double
 // buffered with a CTA barrier per slice.  In both the weight stream does not depend on the preceding kernel, so it
 // is started before the grid dependency is awaited.  q4_gemm_kernel is the older CTA-granular form (a CTA owns 128
 // rows and one K-slice, split-K through global scratch); the grouped mode of the mixture-of-experts layers still
@@ -448,10 +448,9 @@ __device__ __forceinline__ void tile_epilogue(const Params& p, const float (&acc
 }
 
 // ---- round kernel ------------------------------------------------------------------------------------------------
-// One CTA of 8 warps per SM owns a contiguous range of row tiles (MT sub-tiles of 16 rows each, so that the
-// activation fragments a warp reads from shared memory serve 16 MT rows: the multiply loop is bound by shared-memory
-// wavefronts, most of them activation reads) and one part of K (at most four slices of 1024 input features; most
-// projections have a single part).  It walks its tiles in rounds of at most 8 / kw tiles; kw warps share a tile
+// One CTA of kRoundWarps warps per SM owns a contiguous range of row tiles (of 16 rows) and one part of K (at most
+// four slices of 1024 input features; most projections have a single part).  It walks its tiles in rounds of at
+// most kRoundWarps / kw tiles; kw warps share a tile
 // (stage j of the tile's stages goes to warp j mod kw of the tile) and add their accumulators through shared
 // memory at the end of the round.  The CTA moves through the slices together: the activations of the
 // next slice arrive by bulk copy in the other of two buffers while the warps multiply the current one, with one CTA
@@ -480,7 +479,9 @@ struct RoundParams {
 };
 
 constexpr int kRoundMT = 1;  // sub-tiles of 16 rows per warp tile (2, with 8 warps of 198 registers, measured no faster)
-constexpr int kRoundWarps = 16 / kRoundMT, kRoundThreads = 32 * kRoundWarps;
+// 12 warps of up to 170 registers: with 16 the 128-register cap cost more in instruction scheduling than the four
+// extra warps gave (LM head 175 -> 138 us, the batch-1 step of the 8B shape 3.00 -> 2.70 ms)
+constexpr int kRoundWarps = 12, kRoundThreads = 32 * kRoundWarps;
 // a stage: 16 MT rows of 128 B of codes, 16-byte chunks swizzled by row, then the rows' scales and biases
 constexpr int kRoundRows = 16 * kRoundMT, kRoundStage = kRoundRows * (128 + kSbBytes);
 
@@ -812,9 +813,9 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   }
 }
 
-// ---- span kernel: projections whose CTAs hold at most 16 row tiles ------------------------------------------------
+// ---- span kernel: projections whose CTAs hold at most kRoundWarps row tiles ---------------------------------------
 // All K-slices of the CTA's part of K (at most four) are resident in shared memory, so nothing ties the warps to one
-// another while they multiply.  The CTA's stages, row tile major, are cut into 16 equal contiguous spans, one per
+// another while they multiply.  The CTA's stages, row tile major, are cut into equal contiguous spans, one per
 // warp: every warp streams the same number of stages (to within one) whatever the number of tiles, a span covers the
 // tail of one tile and the head of the next at most, and each warp refills the ring slot it has just multiplied.
 // At the end the warps leave their (one or two) partial sums in shared memory, and the warp that holds a tile's first
@@ -917,9 +918,9 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
   // the CTA's tiles, and this warp's span of their stages
   const int t0 = (int)((long long)blockIdx.x * p.T / gridDim.x), t1 = (int)((long long)(blockIdx.x + 1) * p.T / gridDim.x);
   const int Tc = t1 - t0, Lc = Tc * SQ;
-  // Span i belongs to warp (i % 4) * 4 + i / 4: when only every second or fourth span holds a stage (few stages per
+  // Span (w % 4) * (W / 4) + w / 4 belongs to warp w: when only every second or fourth span holds a stage (few stages per
   // CTA) the busy warps still spread over the four schedulers of the SM.
-  const int span = (warp & 3) * 4 + (warp >> 2);
+  const int span = (warp & 3) * (W / 4) + (warp >> 2);
   auto span_begin = [&](int i) -> int { return i * Lc / W; };
   const int a = span_begin(span), cnt = span_begin(span + 1) - a;
   const int tlA = a / SQ, jA0 = a - tlA * SQ;
@@ -1141,7 +1142,7 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   // two ring slots per warp (every slot is refilled as soon as it is multiplied); four for <= 8 requests and
   // long K, where the operand is half the size and the multiply loop shorter.  Small footprints matter: the next
   // projection's CTAs can then become resident, and request their weights, before this one has left the SM.
-  t.span_stages = (t.nt == 1 && t.S >= 3) ? 4 : 2;
+  t.span_stages = t.S >= 3 ? (t.nt == 1 ? 4 : (t.S >= 4 ? 3 : 2)) : 2;
   const size_t operand = t.S * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   const size_t handover = (size_t)kRoundWarps * 2 * 16 * np * sizeof(float);  // two partial tiles per warp, in the operand's place
   t.span_smem = (size_t)kRoundWarps * t.span_stages * kRoundStage + (operand > handover ? operand : handover);
@@ -1273,6 +1274,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   if (const char* f = getenv("Q4D_GEMM_PART_SLICES")) g_part_slices = atoi(f) < 1 ? 1 : (atoi(f) > 4 ? 4 : atoi(f));
@@ -1306,6 +1308,7 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     if (t.span) {
       if (t.nt == 1 && t.span_stages == 2) return launch_kernel(q4_span_kernel<1, 2>, grid, block, t.span_smem, s, p);
       if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 4>, grid, block, t.span_smem, s, p);
+      if (t.span_stages == 3) return launch_kernel(q4_span_kernel<2, 3>, grid, block, t.span_smem, s, p);
       return launch_kernel(q4_span_kernel<2, 2>, grid, block, t.span_smem, s, p);
     }
     if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
