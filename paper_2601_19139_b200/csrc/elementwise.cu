@@ -26,7 +26,16 @@ __global__ void embed_kernel(const uint32_t* q, const uint16_t* scales, const ui
   const uint32_t* qrow = q + (size_t)tok * (H >> 3);
   const uint16_t* srow = scales + (size_t)tok * (H >> 6);
   const uint16_t* brow = biases + (size_t)tok * (H >> 6);
-  for (int k = threadIdx.x; k < H; k += blockDim.x) x[(size_t)r * H + k] = f32_to_bf16(dequant(qrow, srow, brow, k));
+  // one packed word (8 elements) per thread and pass: its three loads go out together, one 16-byte store
+  for (int w8 = threadIdx.x; w8 < (H >> 3); w8 += blockDim.x) {
+    const uint32_t word = qrow[w8];
+    const float sc = bf16_to_f32(srow[w8 >> 3]), bi = bf16_to_f32(brow[w8 >> 3]);
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      o[j] = pack_bf16x2(__fmaf_rn(sc, (float)((word >> (8 * j)) & 0xFu), bi), __fmaf_rn(sc, (float)((word >> (8 * j + 4)) & 0xFu), bi));
+    *reinterpret_cast<uint4*>(x + (size_t)r * H + w8 * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
 }
 
 __device__ __forceinline__ float block_sum(float v, float* red) {
