@@ -132,6 +132,19 @@ def oracle_sample(shape, weights, pool_t, lens, toks, bt, budget_layers):
     return full, desc, orc.num_threads()
 
 
+def aggregate_ranks(dist, device, ms, ms_e2e, tokens, tokens_e2e, launches):
+    """Replicas only: every rank ran its own batch.  The job's time is the slowest rank's, its tokens and kernel
+    launches are the sums over the ranks.  `dist` is torch.distributed with an initialised process group, or None."""
+    if dist is None:
+        return ms, ms_e2e, tokens, tokens_e2e, launches
+    import torch
+    t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    c = torch.tensor([tokens, tokens_e2e, launches], dtype=torch.float64, device=device)
+    dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), int(c[0]), int(c[1]), int(c[2])
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -354,13 +367,7 @@ def main():
                     "timing": "CUDA events around each launch, profile pass right after the timed steps"}
 
     # ---- max over ranks, aggregate ----
-    if dist is not None:
-        t = torch.tensor([ms, ms_e2e], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
-        c = torch.tensor([tokens, tokens_e2e, launches], dtype=torch.float64, device=device)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tokens, tokens_e2e, launches = int(c[0]), int(c[1]), int(c[2])
+    ms, ms_e2e, tokens, tokens_e2e, launches = aggregate_ranks(dist, device, ms, ms_e2e, tokens, tokens_e2e, launches)
 
     value = tokens / (ms * 1e-3)
     step_gbs = mean_bytes["total"] / (ms / args.steps * 1e-3) / 1e9
