@@ -1139,9 +1139,10 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
   t.span = per_cta <= kRoundWarps && kRoundMT == 1;
-  // two ring slots per warp (every slot is refilled as soon as it is multiplied); four for <= 8 requests and
-  // long K, where the operand is half the size and the multiply loop shorter.  Small footprints matter: the next
-  // projection's CTAs can then become resident, and request their weights, before this one has left the SM.
+  // Ring slots per warp (every slot is refilled as soon as it is multiplied): two for short K, where a small
+  // footprint lets the next projection's CTAs become resident, and request their weights, before this one has left
+  // the SM; with four slices resident, three (what fits) for 9-16 requests and four for <= 8 requests, whose operand
+  // is half the size and whose multiply loop is shorter.
   t.span_stages = t.S >= 3 ? (t.nt == 1 ? 4 : (t.S >= 4 ? 3 : 2)) : 2;
   const size_t operand = t.S * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   const size_t handover = (size_t)kRoundWarps * 2 * 16 * np * sizeof(float);  // two partial tiles per warp, in the operand's place
