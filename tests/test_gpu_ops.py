@@ -93,6 +93,46 @@ def test_q4_gemm_bf16_and_residual_epilogues(q4d):
     assert_bf16_close(bits(res), want_res, what="residual epilogue")
 
 
+def _random_gemm_shapes(count, seed):
+    """Seeded shapes that land in every branch of the projection kernels' planning: one tile or thousands, spans
+    shorter than a stage or several tiles long, one to twelve K-slices (K up to three parts), both batch classes."""
+    rng = np.random.default_rng(seed)
+    shapes_ = []
+    for _ in range(count):
+        N = int(rng.choice([rng.integers(1, 64), rng.integers(64, 2400), rng.integers(2400, 30000)]))
+        K = 256 * int(rng.choice([1, 2, 3, 4, 5, 8, 12, 16, 20, 48]))
+        if N * K > 40_000_000:
+            N = 40_000_000 // K
+        shapes_.append((N, K, int(rng.integers(1, 17)), int(rng.integers(0, 3))))
+    return shapes_
+
+
+@pytest.mark.parametrize("N,K,n,epi", _random_gemm_shapes(14, 2024))
+def test_q4_gemm_random_shapes_every_epilogue(q4d, N, K, n, epi):
+    w = gen.random_q4(N, K, "cuda", "gpu-gemm-rand", N, K)
+    x = _rand_bf16((n, K), N + 3 * K + n)
+    want = orc.q4_matmul(*_np_triple(w), bits(x))
+    if epi == 2:
+        got = q4d.q4_gemm(w, x, n, epilogue=2).cpu().numpy().astype(np.float64)
+        rms = np.sqrt((want ** 2).mean())
+        assert np.abs(got - want).max() <= 3e-5 * rms, np.abs(got - want).max() / rms
+    elif epi == 0:
+        assert_bf16_close(bits(q4d.q4_gemm(w, x, n, epilogue=0)), orc.bf16_round(want), what="bf16 epilogue")
+    else:
+        res = _rand_bf16((n, N), N + K, 0.5)
+        res_in = bits(res).copy()
+        q4d.q4_gemm(w, x, n, epilogue=1, out=res)
+        v = orc.bf16_to_f64(orc.bf16_round(want))
+        want_res = orc.bf16_to_f64(orc.bf16_round(orc.bf16_to_f64(res_in) + v))
+        got_res = orc.bf16_to_f64(bits(res))
+        # bf16(v) may land one step of v apart (fp32 vs fp64 sums next to a rounding boundary); where the residual
+        # cancels v that step is several steps of the sum, so the bound is a step of v plus a step of the sum
+        step = lambda a: 2.0 ** (np.floor(np.log2(np.maximum(np.abs(a), 1e-30))) - 7)
+        err = np.abs(got_res - want_res)
+        assert (err <= step(v) + step(want_res)).all(), float((err / (step(v) + step(want_res))).max())
+        assert (got_res != want_res).mean() <= 0.01
+
+
 def test_q4_gemm_silu_mul_prologue(q4d):
     N, K, n = 1024, 3072, 16
     w = gen.random_q4(N, K, "cuda", "gpu-gemm-silu")
