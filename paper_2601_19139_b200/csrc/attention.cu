@@ -460,16 +460,17 @@ AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, i
     chunk_tiles = (chunk_tokens + 15) / 16;
   } else {
     // One wave: two CTAs fit on an SM, so aim at 2 * sm_count items of equal size (a multiple of 4 tiles so
-    // that the four warps of a CTA get equal shares), at least 4 tiles and at most 64.
+    // that the four warps of a CTA get equal shares), at least 4 tiles and at most 512: a second, partly filled
+    // wave of shorter items costs more than one wave of longer ones.
     const long long slots = 2LL * sm_count;
     long long ct = (total_tiles * nkv + slots - 1) / slots;
     ct = (ct + 3) / 4 * 4;
-    chunk_tiles = (int)(ct < 4 ? 4 : (ct > 64 ? 64 : ct));
+    chunk_tiles = (int)(ct < 4 ? 4 : (ct > 512 ? 512 : ct));
     // requests add a ragged last chunk each: grow the chunk until the items fit the wave
     for (;;) {
       long long items = 0;
       for (int r = 0; r < n; ++r) items += ((lens[r] + 1 + 15) / 16 + chunk_tiles - 1) / chunk_tiles;
-      if (items * nkv <= slots || chunk_tiles >= 64) break;
+      if (items * nkv <= slots || chunk_tiles >= 512) break;
       chunk_tiles += 4;
     }
   }
