@@ -350,7 +350,7 @@ def main():
         class_kernel = {"attention": "paged_attention_kernel", "lm_head": "q4_round_kernel", "moe_gate_up": "q4_gemm_kernel", "moe_down": "q4_gemm_kernel"}
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped
         # batch-16 case (see profiles/); traffic is proportional to the bytes streamed, so it is scaled to this launch.
-        traffic_ratio = {"gemm_gate_up": 1.005, "attention": 1.005}
+        traffic_ratio = {"gemm_gate_up": 1.005, "attention": 1.032}
         total_prof_ms = sum(v[0] for v in prof.values())
         kernels = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
                        "share": v[0] / total_prof_ms} for k, v in prof.items() if v[1]}
