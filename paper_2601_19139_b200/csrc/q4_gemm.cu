@@ -1112,7 +1112,7 @@ struct RoundPlan {
 RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   RoundPlan t;
   t.nt = n <= 8 ? 1 : 2;
-  t.stages = t.nt == 1 ? 5 : 4;
+  t.stages = t.nt == 1 ? 3 : 2;  // ring slots per warp; deeper rings measured slower (LM head: 4 -> 142 us, 5 -> 171 us, 2 -> 137 us)
   const int quads = K / 256;
   t.Q = 1;
   for (int c = kMaxQuadsPerSlice; c >= 1; --c)
@@ -1139,11 +1139,10 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   t.smem = (size_t)kRoundWarps * t.stages * kRoundStage + 2 * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   t.partial_bytes = t.parts > 1 ? (size_t)t.parts * t.T * kRoundRows * np * sizeof(float) : 0;
   t.span = per_cta <= kRoundWarps && kRoundMT == 1;
-  // Ring slots per warp (every slot is refilled as soon as it is multiplied): two for short K, where a small
-  // footprint lets the next projection's CTAs become resident, and request their weights, before this one has left
-  // the SM; with four slices resident, three (what fits) for 9-16 requests and four for <= 8 requests, whose operand
-  // is half the size and whose multiply loop is shorter.
-  t.span_stages = t.S >= 3 ? (t.nt == 1 ? 4 : (t.S >= 4 ? 3 : 2)) : 2;
+  // Two ring slots per warp, each refilled as soon as it is multiplied.  Measured: deeper rings are slower (8B shape,
+  // batch 16, three slots instead of two: gate/up 29 -> 37 us, down 23 -> 27 us) — more requests in flight than the
+  // memory system serves well, and a larger footprint keeps the next projection's CTAs off the SM for longer.
+  t.span_stages = 2;
   const size_t operand = t.S * ((size_t)np * (t.Q * 512 + 16) + (size_t)t.Q * 4 * 16 * 4);
   const size_t handover = (size_t)kRoundWarps * 2 * 16 * np * sizeof(float);  // two partial tiles per warp, in the operand's place
   t.span_smem = (size_t)kRoundWarps * t.span_stages * kRoundStage + (operand > handover ? operand : handover);
@@ -1269,13 +1268,11 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<1, 5>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<1, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+    e = cudaFuncSetAttribute(q4_round_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   if (const char* f = getenv("Q4D_GEMM_PART_SLICES")) g_part_slices = atoi(f) < 1 ? 1 : (atoi(f) > 4 ? 4 : atoi(f));
@@ -1307,13 +1304,11 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
     const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
     if (t.span) {
-      if (t.nt == 1 && t.span_stages == 2) return launch_kernel(q4_span_kernel<1, 2>, grid, block, t.span_smem, s, p);
-      if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 4>, grid, block, t.span_smem, s, p);
-      if (t.span_stages == 3) return launch_kernel(q4_span_kernel<2, 3>, grid, block, t.span_smem, s, p);
+      if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 2>, grid, block, t.span_smem, s, p);
       return launch_kernel(q4_span_kernel<2, 2>, grid, block, t.span_smem, s, p);
     }
-    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 5>, grid, block, t.smem, s, p);
-    return launch_kernel(q4_round_kernel<2, 4>, grid, block, t.smem, s, p);
+    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 3>, grid, block, t.smem, s, p);
+    return launch_kernel(q4_round_kernel<2, 2>, grid, block, t.smem, s, p);
   }
   const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;
