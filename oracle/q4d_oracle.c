@@ -195,13 +195,11 @@ void orc_dequant_q4(const uint32_t* q, const uint16_t* scales, const uint16_t* b
     for (int64_t k = 0; k < K; ++k) out[j * K + k] = dequant_one(&t, K, j, k);
 }
 
-/* Sensitivity probe, off by default and never part of the definition: when set, the
- * projections accumulate in fp32 instead of fp64.  Tests use it to measure how far any
- * fp32-accumulating implementation can drift from the fp64 definition once bf16
- * rounding decisions start to differ. */
-static int g_probe_fp32_accumulate = 0;
-void orc_probe_fp32_accumulate(int on) { g_probe_fp32_accumulate = on; }
-
+/* The definition accumulates in fp64.  A second build of this file with
+ * -DORC_SENSITIVITY_PROBE_FP32 (made and loaded only by tests/fp32_probe.py, never by
+ * oracle/build.py) accumulates the projections in fp32 instead: the tests use that
+ * variant to measure how far any fp32-accumulating implementation drifts from the
+ * definition once bf16 rounding decisions start to differ.  It is not the oracle. */
 /* out[r][j] = sum_k w[j][k] * x[r][k], k ascending, fp64, for rows j in
  * [row0, row0+N) of a tensor with K input features.  x is bf16 [n][K]. */
 static int q4_matmul_rows(const orc_qtensor* t, int64_t row0, int64_t N, int64_t K,
@@ -223,18 +221,18 @@ static int q4_matmul_rows(const orc_qtensor* t, int64_t row0, int64_t N, int64_t
       for (int64_t j = 0; j < N; ++j) {
         for (int64_t k = 0; k < K; ++k) wrow[k] = dequant_one(t, K, row0 + j, k);
         for (int32_t r = 0; r < n; ++r) acc[r] = 0.0;
-        if (g_probe_fp32_accumulate) {
-          for (int64_t k = 0; k < K; ++k) {
-            const double* xk = xt + k * n;
-            for (int32_t r = 0; r < n; ++r) acc[r] = (double)((float)acc[r] + wrow[k] * (float)xk[r]);
-          }
-        } else {
-          for (int64_t k = 0; k < K; ++k) {
-            double wk = (double)wrow[k];
-            const double* xk = xt + k * n;
-            for (int32_t r = 0; r < n; ++r) acc[r] += wk * xk[r];
-          }
+#ifdef ORC_SENSITIVITY_PROBE_FP32
+        for (int64_t k = 0; k < K; ++k) {
+          const double* xk = xt + k * n;
+          for (int32_t r = 0; r < n; ++r) acc[r] = (double)((float)acc[r] + wrow[k] * (float)xk[r]);
         }
+#else
+        for (int64_t k = 0; k < K; ++k) {
+          double wk = (double)wrow[k];
+          const double* xk = xt + k * n;
+          for (int32_t r = 0; r < n; ++r) acc[r] += wk * xk[r];
+        }
+#endif
         for (int32_t r = 0; r < n; ++r) out[(int64_t)r * out_stride + j] = acc[r];
       }
     }

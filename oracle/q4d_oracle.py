@@ -41,18 +41,21 @@ class Weights(C.Structure):
                 ("lm_head", QTensor), ("rope_cos_sin", C.c_void_p)]
 
 
+def _declare(L):
+    L.orc_bf16_round.restype = C.c_uint16
+    L.orc_bf16_round.argtypes = [C.c_double]
+    L.orc_bf16_to_float.restype = C.c_float
+    L.orc_bf16_to_float.argtypes = [C.c_uint16]
+    L.orc_num_threads.restype = C.c_int
+    for name in ("orc_q4_matmul", "orc_attention_head", "orc_attention_paged", "orc_decode_step"):
+        getattr(L, name).restype = C.c_int
+    return L
+
+
 def lib():
     global _LIB
     if _LIB is None:
-        L = C.CDLL(_build.build())
-        L.orc_bf16_round.restype = C.c_uint16
-        L.orc_bf16_round.argtypes = [C.c_double]
-        L.orc_bf16_to_float.restype = C.c_float
-        L.orc_bf16_to_float.argtypes = [C.c_uint16]
-        L.orc_num_threads.restype = C.c_int
-        for name in ("orc_q4_matmul", "orc_attention_head", "orc_attention_paged", "orc_decode_step"):
-            getattr(L, name).restype = C.c_int
-        _LIB = L
+        _LIB = _declare(C.CDLL(_build.build()))
     return _LIB
 
 
@@ -202,11 +205,6 @@ def attention_paged(q_bits, pool, nq, nkv, bs, d, layer, lens, block_tables):
                                    _p(bt), C.c_int32(bt.shape[1]), _p(out))
     assert rc == 0, rc
     return out
-
-
-def probe_fp32_accumulate(on):
-    """Sensitivity probe (not the definition): projections accumulate in fp32 while set."""
-    lib().orc_probe_fp32_accumulate(C.c_int(int(bool(on))))
 
 
 def num_threads():

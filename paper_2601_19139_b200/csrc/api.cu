@@ -544,6 +544,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   float* logits = logits_dev ? logits_dev : at<float>(m, m->lay.logits);
   const size_t layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
   const int qdim = nq * kHeadDim;
+  const int dense_layout = gemm_operand_layout(false);  // of the operands of the dense projections
 
 #define Q4D_LAUNCH(cls, expr)                                                 \
   do {                                                                        \
@@ -561,7 +562,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     const q4d_layer_weights& lw = m->layers[l];
     uint16_t* kpool = pool->mem + (size_t)(2 * l) * layer_elems;
     uint16_t* vpool = kpool + layer_elems;
-    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+    Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.attn_norm, sh.rms_eps, n, H, nullptr, yp, ys, dense_layout, s));
     Q4D_LAUNCH(Q4D_K_GEMM_QKV, launch_q4_gemm(gemm_args(m, lw.wqkv, nqkv, H, yp, ys, n, EPI_BF16, qkv, nqkv), s));
     AttnArgs aa;
     aa.q = qbuf, aa.kpool = kpool, aa.vpool = vpool, aa.block_tables = d_bt, aa.lens = d_lens;
@@ -570,7 +571,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     aa.nchunks = reinterpret_cast<const int32_t*>(dmeta + ml.off_nchunks);
     aa.n_work = plan.n_work, aa.n = n, aa.nq = nq, aa.nkv = nkv, aa.max_blocks = ml.max_blocks_cap;
     aa.part_acc = at<float>(m, m->lay.part_acc), aa.part_ml = at<float>(m, m->lay.part_ml);
-    aa.out = nullptr, aa.out_xp = ap, aa.out_xs = as;
+    aa.out = nullptr, aa.out_xp = ap, aa.out_xs = as, aa.out_layout = dense_layout;
     aa.merge_counters = at<int>(m, m->lay.attn_merge_counters);  // the last CTA of a (request, kv head) merges its chunks
     // q preparation (qk-norm, rotary embedding) and the append of k, v happen inside the attention kernel
     aa.qkv = qkv, aa.q_norm = sh.qk_norm ? lw.q_norm : nullptr, aa.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
@@ -578,11 +579,11 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
     Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
     if (sh.n_experts == 0) {
-      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, nullptr, yp, ys, dense_layout, s));
       GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
       gu.out_xp = hp, gu.out_xs = hs;
       Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
-      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, nullptr, n, EPI_RESIDUAL, x, H), s));
+      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
     } else {
       const int E = sh.n_experts, Ie = sh.expert_inter;
       uint16_t* yplain = at<uint16_t>(m, m->lay.yplain);
@@ -595,7 +596,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       uint16_t* ehp = at<uint16_t>(m, m->lay.m_hp);
       float* ehs = at<float>(m, m->lay.m_hs);
       uint16_t* eo = at<uint16_t>(m, m->lay.m_o);
-      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, yplain, yp, ys, s));
+      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, yplain, yp, ys, gemm_operand_layout(true), s));
       Q4D_LAUNCH(Q4D_K_MOE_ROUTER, launch_moe_router(mr, n, s));
       GemmArgs gu = gemm_args(m, lw.experts_gate_up, 2 * Ie, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
       gu.out_xp = ehp, gu.out_xs = ehs;
@@ -616,7 +617,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     cudaError_t ce = cudaMemcpyAsync(range->x_out, x, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
     return ce == cudaSuccess ? Q4D_OK : fail_cuda(ce, "hidden state copy");
   }
-  Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, nullptr, yp, ys, s));
+  Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, nullptr, yp, ys, dense_layout, s));
   GemmArgs lm = gemm_args(m, m->w.lm_head, V, H, yp, ys, n, EPI_F32, logits, V);
   lm.argmax_partial = amax;
   const int lm_blocks = gemm_row_blocks(V, H, n, EPI_F32);
@@ -954,7 +955,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
   uint16_t* xp = reinterpret_cast<uint16_t*>(sc + kOpPackOff);
   float* xs = reinterpret_cast<float*>(sc + kOpPackOff + kOpPackXp);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaError_t e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, st);
+  cudaError_t e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false), st);
   if (e != cudaSuccess) return fail_cuda(e, "q4_gemm (operand)");
   GemmArgs a;
   a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;
@@ -969,7 +970,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
 int q4d_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int32_t n, int32_t H, uint16_t* y, void* stream) {
   if (!x || !w || !y || n < 0 || H < 64 || H % 64 || H > 16384)
     return fail(Q4D_ERR_INVALID_ARG, "rmsnorm: bad argument (H must be a multiple of 64, at most 16384)");
-  cudaError_t e = launch_rmsnorm(x, w, eps, n, H, y, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_rmsnorm(x, w, eps, n, H, y, nullptr, nullptr, OPERAND_ROWS, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "rmsnorm");
 }
 

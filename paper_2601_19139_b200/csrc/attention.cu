@@ -68,7 +68,7 @@ __device__ __forceinline__ void merge_head_chunk(const AttnArgs& p, int r, int a
   const size_t K = (size_t)p.nq * kHeadDim;
   if (p.out) *reinterpret_cast<uint4*>(p.out + (size_t)r * K + col) = o;
   if (p.out_xp) {
-    *reinterpret_cast<uint4*>(p.out_xp + (size_t)r * K + col) = permute_chunk(o);
+    *reinterpret_cast<uint4*>(p.out_xp + operand_chunk_offset(p.out_layout, (int)K, r, (int)(col >> 3))) = permute_chunk(o);
     if ((ch & 7) == 0) p.out_xs[(col >> 6) * 16 + r] = gsum;
   }
 }

@@ -78,6 +78,11 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 // {0,4,1,5,2,6,3,7} (so that a lane's 16 bytes are its B fragments of two k-steps), plus the fp32 sum of every
 // group of 64 elements, [K/64][16].  Producers build both with these helpers, always with the same summation
 // tree: ((e0+e1)+(e2+e3))+((e4+e5)+(e6+e7)) per chunk, then a pairwise tree over the 8 chunks of the group.
+// Element offset of chunk c (8 features) of request r in an operand of K features: layout 0 is [16][K], layout 1 is
+// [K/8][16][8] (all requests of a chunk side by side: the tensor-core kernel copies a K-range as one block).
+__device__ __forceinline__ size_t operand_chunk_offset(int layout, int K, int r, int c) {
+  return layout ? ((size_t)c * 16 + r) * 8 : (size_t)r * K + (size_t)c * 8;
+}
 __device__ __forceinline__ uint4 permute_chunk(const uint4 v) {
   uint4 o;
   o.x = __byte_perm(v.x, v.z, 0x5410);

@@ -52,7 +52,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // y = bf16(x / sqrt(mean(x^2) + eps) * w); one CTA per request row.  The row is held in registers (up to 8 chunks
 // of 8 elements per thread: H <= 16384).  Writes y in plain layout and/or as the next GEMM's operand.
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* x, const uint16_t* w, float eps, int H,
-                                                       uint16_t* y, uint16_t* yp, float* ys) {
+                                                       uint16_t* y, uint16_t* yp, float* ys, int layout) {
   __shared__ float red[8];
   grid_launch_dependents();
   const int r = blockIdx.x, nch = H >> 3;
@@ -96,7 +96,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* x, const u
     if (c < nch) {
       if (y) *reinterpret_cast<uint4*>(y + (size_t)r * H + c * 8) = v;
       if (yp) {
-        *reinterpret_cast<uint4*>(yp + (size_t)r * H + c * 8) = permute_chunk(v);
+        *reinterpret_cast<uint4*>(yp + operand_chunk_offset(layout, H, r, c)) = permute_chunk(v);
         if ((c & 7) == 0) ys[(size_t)(c >> 3) * 16 + r] = gsum;
       }
     }
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const uint16_t* x, const u
 // Plain activations -> the GEMM's fragment-ordered operand (optionally h = bf16(silu(gate) * up) first).
 // One thread per chunk of 8 elements; x is [n][x_stride] (with the SiLU prologue: gate at [0, K), up at [K, 2K)).
 __global__ void __launch_bounds__(256) pack_operand_kernel(const uint16_t* x, int x_stride, int K, int n, int prologue,
-                                                            uint16_t* xp, float* xs) {
+                                                            uint16_t* xp, float* xs, int layout) {
   grid_launch_dependents();
   grid_dependency_wait();
   const int cpr = K >> 3;
@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(256) pack_operand_kernel(const uint16_t* x, in
   }
   const float gsum = group_sum_8lanes(chunk_sum(v));
   if (r < n) {
-    *reinterpret_cast<uint4*>(xp + (size_t)r * K + kc * 8) = permute_chunk(v);
+    *reinterpret_cast<uint4*>(xp + operand_chunk_offset(layout, K, r, kc)) = permute_chunk(v);
     if ((kc & 7) == 0) xs[(size_t)(kc >> 3) * 16 + r] = gsum;
   }
 }
@@ -203,19 +203,19 @@ cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16
 }
 
 cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int n, int H, uint16_t* y,
-                           uint16_t* yp, float* ys, cudaStream_t s) {
+                           uint16_t* yp, float* ys, int layout, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   if (H % 64 || H > 16384 || (yp && !ys)) return cudaErrorInvalidValue;
-  return launch_kernel(rmsnorm_kernel, dim3(n), dim3(256), 0, s, x, w, eps, H, y, yp, ys);
+  return launch_kernel(rmsnorm_kernel, dim3(n), dim3(256), 0, s, x, w, eps, H, y, yp, ys, layout);
 }
 
 cudaError_t launch_pack_operand(const uint16_t* x, int x_stride, int K, int n, int prologue, uint16_t* xp, float* xs,
-                                cudaStream_t s) {
+                                int layout, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   if (K % 256 || x_stride % 8) return cudaErrorInvalidValue;
   const int chunks = n * (K >> 3);
   return launch_kernel(pack_operand_kernel, dim3((chunks + 255) / 256), dim3(256), 0, s, x, x_stride, K, n, prologue,
-                       xp, xs);
+                       xp, xs, layout);
 }
 
 cudaError_t launch_argmax(const float* logits, int n, int vocab, int32_t* next, cudaStream_t s) {

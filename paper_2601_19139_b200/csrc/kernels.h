@@ -19,9 +19,13 @@ bool pdl_enabled();
 
 // ---- fragment-ordered GEMM operand ---------------------------------------------------
 // xp bf16 [16][K] (chunks of 8 permuted), xs f32 [K/64][16] (group sums); see common.cuh.
+// Two layouts of the bf16 elements exist: OPERAND_ROWS, [16][K] (the mma.sync kernels), and OPERAND_BLOCKED,
+// [K/8][16][8] (the tcgen05 kernel: a K-range of all requests is one contiguous block that the tensor core reads as
+// 8-request x 16-byte core matrices).  Both keep the order 0,4,1,5,2,6,3,7 inside a chunk of 8.
 enum GemmPrologue { PRO_PLAIN = 0, PRO_SILU_MUL = 1 };
+enum OperandLayout { OPERAND_ROWS = 0, OPERAND_BLOCKED = 1 };
 cudaError_t launch_pack_operand(const uint16_t* x, int x_stride, int K, int n, int prologue, uint16_t* xp, float* xs,
-                                cudaStream_t s);
+                                int layout, cudaStream_t s);
 
 // ---- 4-bit skinny GEMM ------------------------------------------------------------
 // EPI_SILU_PACK: the tensor has 2*I rows (gate rows then up rows); the output is the operand of the next GEMM,
@@ -60,6 +64,17 @@ size_t gemm_partial_bytes(int N, int K, int epilogue);
 int gemm_counters_needed(int N);
 int gemm_row_blocks(int N, int K, int n, int epilogue);  // grid.x of the launch (size of argmax_partial)
 cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s);
+// The operand layout launch_q4_gemm expects for this call (grouped: the mixture-of-experts mode).
+int gemm_operand_layout(bool grouped);
+
+// tcgen05 kernel (q4_umma.cu): tiles of 128 rows, K in `parts` across CTAs, stages of 256 features.
+struct UmmaPlan {
+  int tiles, parts, ns;
+  size_t partial_bytes;
+};
+UmmaPlan plan_umma(int N, int K, int epilogue, int sm_count);
+bool umma_supported(int N, int K, int epilogue);
+cudaError_t launch_q4_umma(const GemmArgs& a, int sm_count, cudaStream_t s);
 cudaError_t gemm_init();  // sets the dynamic shared memory limits once per process/device
 cudaError_t launch_argmax_finish(const float2* partial, int row_blocks, int n, int32_t* next, cudaStream_t s);
 
@@ -89,6 +104,7 @@ struct AttnArgs {
   uint16_t* out;    // plain [n][nq][128], or NULL
   uint16_t* out_xp; // fragment-ordered operand [16][nq*128] of the O projection, or NULL
   float* out_xs;    // its group sums [nq*2][16]
+  int out_layout = OPERAND_ROWS;  // layout of out_xp
   int* merge_counters = nullptr;  // [16][nkv], zero between launches: the attention kernel merges the chunks itself
   // With qkv given (bf16 [n][(nq+2nkv)*128], the QKV projection's output) the kernel prepares q itself (qk-norm,
   // rotary embedding) and appends k, v of the new token to the pool; `q` is then unused.
@@ -149,7 +165,7 @@ cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16
                          const int32_t* tokens, int n, uint16_t* x, cudaStream_t s);
 // y (plain, optional) and/or the fragment-ordered operand (yp, ys) of the next GEMM.
 cudaError_t launch_rmsnorm(const uint16_t* x, const uint16_t* w, float eps, int n, int H, uint16_t* y,
-                           uint16_t* yp, float* ys, cudaStream_t s);
+                           uint16_t* yp, float* ys, int layout, cudaStream_t s);
 cudaError_t launch_argmax(const float* logits, int n, int vocab, int32_t* next, cudaStream_t s);
 cudaError_t launch_dequant(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int N, int K,
                            float* out, cudaStream_t s);

@@ -80,7 +80,7 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
   // the activations are first rearranged into the order the GEMM reads them in, inside the same array
   uint16_t* xp = reinterpret_cast<uint16_t*>(base + kCounterBytes + kPartialBytes);
   float* xs = reinterpret_cast<float*>(base + kCounterBytes + kPartialBytes + (size_t)16 * kMaxK * 2);
-  e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, s);
+  e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false), s);
   if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: operand rearrangement failed");
   GemmArgs a;
   a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;

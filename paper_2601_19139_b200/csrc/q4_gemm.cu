@@ -1240,8 +1240,13 @@ __global__ void __launch_bounds__(256) argmax_finish_kernel(const float2* partia
 
 }  // namespace
 
+// Dense projections run on the tcgen05 kernel unless Q4D_GEMM_LEGACY is set (development switch).
+static bool g_legacy = false;
+static bool use_umma(int N, int K, int epilogue) { return !g_legacy && umma_supported(N, K, epilogue); }
+
 size_t gemm_partial_bytes(int N, int K, int epilogue) {
   const int sms = sm_count_or_default();
+  if (use_umma(N, K, epilogue)) return plan_umma(N, K, epilogue, sms).partial_bytes;
   const size_t a = plan_rounds(N, K, 8, epilogue, sms).partial_bytes, b = plan_rounds(N, K, 16, epilogue, sms).partial_bytes;
   return a > b ? a : b;
 }
@@ -1249,8 +1254,14 @@ size_t gemm_partial_bytes(int N, int K, int epilogue) {
 int gemm_counters_needed(int N) { return (N + 15) / 16 + 1; }
 
 int gemm_row_blocks(int N, int K, int n, int epilogue) {
+  if (use_umma(N, K, epilogue)) return plan_umma(N, K, epilogue, sm_count_or_default()).tiles * 4;  // one per warp of a tile
   const RoundPlan t = plan_rounds(N, K, n, epilogue, sm_count_or_default());
   return t.ctas * t.parts * kRoundWarps;  // one argmax partial per warp of the grid
+}
+
+int gemm_operand_layout(bool grouped) {
+  (void)sm_count_or_default();
+  return (grouped || g_legacy) ? OPERAND_ROWS : OPERAND_BLOCKED;
 }
 
 cudaError_t gemm_init() {
@@ -1274,6 +1285,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
+  if (const char* f = getenv("Q4D_GEMM_LEGACY")) g_legacy = f[0] == '1';
   if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
   if (const char* f = getenv("Q4D_GEMM_PART_SLICES")) g_part_slices = atoi(f) < 1 ? 1 : (atoi(f) > 4 ? 4 : atoi(f));
   g_sm_count = sms;
@@ -1290,6 +1302,7 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
   const bool grouped = a.expert_ids != nullptr;
   if (a.epilogue == EPI_SILU_PACK && ((a.N % 16) || !a.out_xp || (grouped && !a.out_xs))) return cudaErrorInvalidValue;
   if (grouped && (a.K > 2048 || !a.n_touched || a.max_slots < 1)) return cudaErrorInvalidValue;
+  if (!grouped && use_umma(a.N, a.K, a.epilogue)) return launch_q4_umma(a, g_sm_count, s);
   if (!grouped) {
     const RoundPlan t = plan_rounds(a.N, a.K, a.n, a.epilogue, g_sm_count);
     RoundParams p;

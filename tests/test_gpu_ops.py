@@ -79,6 +79,19 @@ def test_q4_gemm_f32_matches_oracle(q4d, N, K, n):
     assert np.abs(got - want).max() <= 3e-5 * rms, np.abs(got - want).max() / rms
 
 
+def _assert_residual_close(got_bits, res_in_bits, want):
+    """out = bf16(res + bf16(v)) against the oracle's.  bf16(v) may land one step of v apart (fp32 vs fp64 sums next
+    to a rounding boundary); where the residual cancels v that step is several steps of the sum, so the bound is a
+    step of v plus a step of the sum, and at most 1 % of the elements may differ at all."""
+    v = orc.bf16_to_f64(orc.bf16_round(want))
+    want_res = orc.bf16_to_f64(orc.bf16_round(orc.bf16_to_f64(res_in_bits) + v))
+    got_res = orc.bf16_to_f64(got_bits)
+    step = lambda a: 2.0 ** (np.floor(np.log2(np.maximum(np.abs(a), 1e-30))) - 7)
+    err = np.abs(got_res - want_res)
+    assert (err <= step(v) + step(want_res)).all(), float((err / (step(v) + step(want_res))).max())
+    assert (got_res != want_res).mean() <= 0.01
+
+
 def test_q4_gemm_bf16_and_residual_epilogues(q4d):
     N, K, n = 2048, 1024, 16
     w = gen.random_q4(N, K, "cuda", "gpu-gemm-epi")
@@ -89,8 +102,7 @@ def test_q4_gemm_bf16_and_residual_epilogues(q4d):
     res = _rand_bf16((n, N), 6, 0.5)
     res_in = bits(res).copy()
     q4d.q4_gemm(w, x, n, epilogue=1, out=res)
-    want_res = orc.bf16_round(orc.bf16_to_f64(res_in) + orc.bf16_to_f64(orc.bf16_round(want)))
-    assert_bf16_close(bits(res), want_res, what="residual epilogue")
+    _assert_residual_close(bits(res), res_in, want)
 
 
 def _random_gemm_shapes(count, seed):
@@ -122,15 +134,7 @@ def test_q4_gemm_random_shapes_every_epilogue(q4d, N, K, n, epi):
         res = _rand_bf16((n, N), N + K, 0.5)
         res_in = bits(res).copy()
         q4d.q4_gemm(w, x, n, epilogue=1, out=res)
-        v = orc.bf16_to_f64(orc.bf16_round(want))
-        want_res = orc.bf16_to_f64(orc.bf16_round(orc.bf16_to_f64(res_in) + v))
-        got_res = orc.bf16_to_f64(bits(res))
-        # bf16(v) may land one step of v apart (fp32 vs fp64 sums next to a rounding boundary); where the residual
-        # cancels v that step is several steps of the sum, so the bound is a step of v plus a step of the sum
-        step = lambda a: 2.0 ** (np.floor(np.log2(np.maximum(np.abs(a), 1e-30))) - 7)
-        err = np.abs(got_res - want_res)
-        assert (err <= step(v) + step(want_res)).all(), float((err / (step(v) + step(want_res))).max())
-        assert (got_res != want_res).mean() <= 0.01
+        _assert_residual_close(bits(res), res_in, want)
 
 
 def test_q4_gemm_silu_mul_prologue(q4d):

@@ -16,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+import fp32_probe
 from gpu_util import Scenario, assert_bf16_close, bits, from_bits, gpu_layer, rel_err
 from oracle import q4d_oracle as orc
 from workload import gen, shapes
@@ -89,8 +90,10 @@ def _run_steps(q4d, sc, steps):
         total += n
         for r in range(n):
             blk, slot = bt[r, sc.lens[r] // 16], sc.lens[r] % 16
-            # layer 0 sees identical inputs on both sides: its appended K, V must match to a bf16 step
-            assert_bf16_close(bits(sc.pool[0, :, blk, :, slot]), sc.host_pool[0, :, blk, :, slot], max_ulp=2,
+            # layer 0 sees identical inputs on both sides: its appended K, V match up to rounding.  A QKV output that
+            # rounds one bf16 step apart (fp32 vs fp64 sums) moves, through the rotation k'_i = k_i c - k_(i+64) s, a
+            # small k'_i by one step of the larger partner: a few steps of k'_i, on a small fraction of elements.
+            assert_bf16_close(bits(sc.pool[0, :, blk, :, slot]), sc.host_pool[0, :, blk, :, slot], max_ulp=8,
                               max_mismatch_frac=0.03, what="layer-0 appended kv")
             sc.pool[:, :, blk, :, slot] = from_bits(sc.host_pool[:, :, blk, :, slot])
             assert pool.request_len(int(ids[r])) == sc.lens[r] + 1
@@ -271,11 +274,8 @@ def _check_against_drift_band(q4d, sc, steps):
     inputs: the GPU's rms logit error must stay within 3x of that drift (and the max within 3x of its max)."""
     bt = sc.block_tables()
     ref = sc.oracle.decode_step(sc.host_pool.copy(), 16, sc.lens, sc.tokens, bt)
-    orc.probe_fp32_accumulate(True)
-    try:
+    with fp32_probe.fp32_accumulation():
         probe = sc.oracle.decode_step(sc.host_pool.copy(), 16, sc.lens, sc.tokens, bt)
-    finally:
-        orc.probe_fp32_accumulate(False)
     pmax, prms = _logit_err(probe[1], ref[1])
     band_max, band_rms = float(pmax.max()), float(prms.max())
     agree, total, worst_max, worst_rms = _run_steps(q4d, sc, steps)
