@@ -19,6 +19,7 @@
 // rows and one K-slice, split-K through global scratch); the grouped mode of the mixture-of-experts layers still
 // runs on it.
 #include <stdlib.h>
+#include <string.h>
 
 #include "common.cuh"
 #include "kernels.h"
@@ -1099,7 +1100,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
   }
 }
 
-int g_part_slices = 4;  // K-slices per part of K; debugging aid: Q4D_GEMM_PART_SLICES
+constexpr int g_part_slices = 4;  // K-slices per part of K
 
 struct RoundPlan {
   int nt, stages, Q, S, parts, T, Tsub, ctas, kw;
@@ -1161,7 +1162,6 @@ struct Tiling {
 };
 
 int g_sm_count = 0;
-int g_force_cfg = -1;  // debugging aid: environment variable Q4D_GEMM_CFG forces the n > 8 configuration
 
 Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count, bool grouped = false) {
   Tiling t;
@@ -1170,12 +1170,8 @@ Tiling choose_tiling(int N, int K, int n, int epilogue, int sm_count, bool group
   if (n <= 8) {
     t.cfg = 0, t.nt = 1, t.rows_cta = 128;
   } else {
-    // 256-row CTAs (one per SM) when they fill the machine, else 128-row CTAs (two per SM)
-    const int rb256 = (rows_logical + 127) / 128 / (epilogue == EPI_SILU_PACK ? 1 : 2);
-    (void)rb256;
     t.cfg = 2;  // two 128-row CTAs per SM hide more latency than one 256-row CTA (measured)
-    if (g_force_cfg == 1 || g_force_cfg == 2) t.cfg = g_force_cfg;
-    t.nt = 2, t.rows_cta = t.cfg == 1 ? 256 : 128;
+    t.nt = 2, t.rows_cta = 128;
   }
   const int rows_per_block = epilogue == EPI_SILU_PACK ? t.rows_cta / 2 : t.rows_cta;
   t.rowblocks = (rows_logical + rows_per_block - 1) / rows_per_block;
@@ -1240,8 +1236,9 @@ __global__ void __launch_bounds__(256) argmax_finish_kernel(const float2* partia
 
 }  // namespace
 
-// Dense projections run on the tcgen05 kernel unless Q4D_GEMM_LEGACY is set (development switch).
-static bool g_legacy = false;
+// Dense projections run on the span/round kernels; Q4D_GEMM_KERNEL=tcgen05 (read once per process) selects the
+// tcgen05 kernel of q4_umma.cu instead, which is correct on every shape but, as measured, not yet faster.
+static bool g_legacy = true;
 static bool use_umma(int N, int K, int epilogue) { return !g_legacy && umma_supported(N, K, epilogue); }
 
 size_t gemm_partial_bytes(int N, int K, int epilogue) {
@@ -1285,9 +1282,7 @@ cudaError_t gemm_init() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e != cudaSuccess) return e;
-  if (const char* f = getenv("Q4D_GEMM_LEGACY")) g_legacy = f[0] == '1';
-  if (const char* f = getenv("Q4D_GEMM_CFG")) g_force_cfg = atoi(f);
-  if (const char* f = getenv("Q4D_GEMM_PART_SLICES")) g_part_slices = atoi(f) < 1 ? 1 : (atoi(f) > 4 ? 4 : atoi(f));
+  if (const char* f = getenv("Q4D_GEMM_KERNEL")) g_legacy = strcmp(f, "tcgen05") != 0;
   g_sm_count = sms;
   return cudaSuccess;
 }
