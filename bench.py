@@ -6,9 +6,10 @@ leaving and four joining (512 prefilled tokens) every 32 steps; `--workload` sel
 
   value      tokens/s with everything resident in HBM (tokens chained on the device, no host sync)
   e2e        tokens/s through q4d_decode_step_host: host inputs, host outputs, a sync per step
-  roofline   the dominant kernel (the launch class with the largest share of the step: a 4-bit projection or the
-             paged attention) timed with CUDA events around each of its launches
-  cpu_baseline  the CPU oracle on a bounded sample of the same step, on the host cores
+  roofline   the dominant kernel (the kernel whose launches take the largest share of the step; the projection
+             kernel serves four launch classes per layer) timed with CUDA events around each of its launches
+  cpu_baseline  the CPU oracle on whole steps of the same workload, on the host cores
+  parity     the last step of the run compared with the oracle (free-running through every layer)
 
 `--impl reference` times the CPU oracle alone (the only reference implementation there is).
 With N > 1 every rank runs an independent replica (requests are independent; there is no exchange).
@@ -92,13 +93,12 @@ class ClockSampler:
                 "samples": len(rows)}
 
 
-def step_bytes(shape, lens, n):
-    """Algorithmic bytes of one step: packed weights + scales + biases, KV read and written, logits, embedding rows."""
+def step_bytes(shape, lens, n, touched=None):
+    """Algorithmic bytes of one step: packed weights + scales + biases, KV read and written, logits, embedding rows.
+    touched: mixture-of-experts models, the mean number of distinct experts per layer the step routes to (measured:
+    q4d_moe_touched_experts); until it is known the expectation under uniform routing stands in."""
     from workload import shapes
-    # mixture of experts: the experts a step touches depend on the routing; the expectation under uniform routing
-    # (E * (1 - (1 - k/E)^n) distinct experts per layer) stands in for the count, which the library does not export
-    touched = None
-    if shape.n_experts:
+    if shape.n_experts and touched is None:
         touched = shape.n_experts * (1.0 - (1.0 - shape.top_k / shape.n_experts) ** n)
     w = shapes.weight_bytes(shape, touched)
     per_tok_layer = 2 * shape.n_kv_heads * shape.head_dim * 2
@@ -110,26 +110,23 @@ def step_bytes(shape, lens, n):
             "total": w + kv_read + kv_write + logits + embed_rows}
 
 
-def oracle_sample(shape, weights, pool_t, lens, toks, bt, budget_layers):
-    """Times the oracle on a bounded sample of one step: the embedding + final norm + LM head alone, then the same
-    with the first `budget_layers` layers; the full-step time is extrapolated by layer count.  Returns
-    (seconds per full step, description, threads)."""
+def oracle_steps(shape, weights, pool_t, lens, toks, bt, max_steps, budget_s):
+    """Times the oracle, as it stands, on whole decode steps of this workload (every layer, the LM head, the
+    argmax): at most max_steps steps, stopping once budget_s seconds are spent.  Every step starts from the same
+    pool.  Returns (seconds per step, steps timed, description, threads, (next tokens, logits) of the step)."""
     from oracle import q4d_oracle as orc
-    Ls = max(1, min(budget_layers, shape.n_layers))
-    sub = dict(weights)
-    sub["layers"] = weights["layers"][:Ls]
-    om = orc.OracleModel(shape, sub)
-    host_pool = orc.to_np(pool_t[:Ls]).copy()
-    t0 = time.perf_counter()
-    om.decode_step(host_pool, 16, lens, toks, bt, layer_limit=0, want_logits=False)
-    t_head = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    om.decode_step(host_pool, 16, lens, toks, bt, layer_limit=Ls, want_logits=False)
-    t_ls = time.perf_counter() - t0
-    full = t_head + (t_ls - t_head) * shape.n_layers / Ls
-    desc = (f"one step of this workload (n={len(lens)}): LM head timed alone ({t_head:.2f} s) and with the first {Ls} "
-            f"of {shape.n_layers} layers ({t_ls:.2f} s); per-step time extrapolated by layer count")
-    return full, desc, orc.num_threads()
+    om = orc.OracleModel(shape, weights)
+    host_pool = orc.to_np(pool_t).copy()
+    times, result = [], None
+    while len(times) < max_steps and (not times or sum(times) + times[-1] < budget_s):
+        work = host_pool.copy()
+        t0 = time.perf_counter()
+        nxt, logits, _ = om.decode_step(work, 16, lens, toks, bt)
+        times.append(time.perf_counter() - t0)
+        result = (nxt, logits)
+    desc = (f"{len(times)} whole decode step(s) of this workload (n={len(lens)}, all {shape.n_layers} layers, LM head, "
+            f"argmax), {np.mean(times):.2f} s each")
+    return float(np.mean(times)), len(times), desc, orc.num_threads(), result
 
 
 def aggregate_ranks(dist, device, ms, ms_e2e, tokens, tokens_e2e, launches):
@@ -153,7 +150,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3-8b-b16", choices=sorted(WORKLOADS))
     ap.add_argument("--profile-steps", type=int, default=8)
-    ap.add_argument("--oracle-layers", type=int, default=4, help="layers in the CPU-baseline sample")
+    ap.add_argument("--oracle-budget", type=float, default=20.0, help="seconds of oracle steps in the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
@@ -203,19 +200,14 @@ def main():
                              f"distinct experts per layer under uniform routing")
 
     if args.impl == "reference":
-        # The reference arm is the CPU oracle: every "step" is the same bounded sample, extrapolated to a full step.
+        # The reference arm is the CPU oracle on whole steps: one warm-up step, then as many of the requested steps
+        # as fit in about two minutes (a step of the 8B shape takes several seconds on the host cores).
         ids, toks, lens, bt = script.step_inputs()
-        times, cores, desc = [], 0, ""
-        for i in range(args.warmup + args.steps):
-            full, desc, cores = oracle_sample(shape, weights, pool_t, lens, toks, bt, args.oracle_layers)
-            if i >= min(args.warmup, 1):
-                times.append(full)
-            if sum(times) > 150 or len(times) >= args.steps:
-                break
-        t = float(np.mean(times))
+        oracle_steps(shape, weights, pool_t, lens, toks, bt, 1, 0.0)
+        t, timed, desc, cores, _ = oracle_steps(shape, weights, pool_t, lens, toks, bt, args.steps, 100.0)
         v = n / t
         print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s", "n_gpus": 0,
-                          "steps": len(times), "warmup": min(args.warmup, 1), "ms_per_step": t * 1e3,
+                          "steps": timed, "warmup": 1, "ms_per_step": t * 1e3,
                           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
                           "data": "synthetic", "config": config,
                           "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
@@ -240,15 +232,18 @@ def main():
                 pool.request_release(ev[1])
 
     bytes_log = []
+    kv_tokens_log = []
+    touched = {"mean": None}    # mean distinct experts per layer a step routes to (measured in the profile pass)
 
-    def one_step(mode):
+    def one_step(mode, want_logits=False):
         """mode 'chained': the fed-in tokens stay on the device; 'host': q4d_decode_step_host."""
         script.churn()
         apply_events()
         ids, toks, lens, bt = script.step_inputs()
-        bytes_log.append(step_bytes(shape, lens, len(ids)))
+        bytes_log.append(step_bytes(shape, lens, len(ids), touched["mean"]))
+        kv_tokens_log.append(float(np.mean(lens)) + 1.0)
         if mode == "host":
-            out, _ = q4d.decode_step_host(model, pool, ids, toks, bt)
+            out, _ = q4d.decode_step_host(model, pool, ids, toks, bt, want_logits=want_logits)
             script.advance(out)
             bufs["rids"] = None
             return len(ids)
@@ -283,6 +278,7 @@ def main():
     barrier()
     launches0 = model.launch_count()
     bytes_log.clear()
+    kv_tokens_log.clear()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
     e0.record(stream)
@@ -295,7 +291,8 @@ def main():
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(wall0, wall1)
     launches = model.launch_count() - launches0
-    mean_bytes = {k: float(np.mean([b[k] for b in bytes_log])) for k in bytes_log[0]}
+    timed_bytes = list(bytes_log)
+    mean_kv_tokens = float(np.mean(kv_tokens_log))
 
     # ---- timed region 2: the same steps through the host-buffer entry point ----
     barrier()
@@ -307,6 +304,15 @@ def main():
     ms_e2e = (time.perf_counter() - t_host0) * 1e3   # every step ends with a stream sync, so host time is device time
     barrier()
     h2d, d2h = model.step_io_bytes()
+    # the same entry point with the logits copied back as well (n x vocab x 4 bytes per step), on fewer steps
+    logit_steps = max(1, min(args.steps, 16))
+    t_host0 = time.perf_counter()
+    tokens_lg = 0
+    for _ in range(logit_steps):
+        tokens_lg += one_step("host", want_logits=True)
+    torch.cuda.synchronize()
+    ms_e2e_lg = (time.perf_counter() - t_host0) * 1e3
+    h2d_lg, d2h_lg = model.step_io_bytes()
 
     # ---- per-launch timing (events around every launch) for the roofline of the dominant kernel ----
     fused = model.is_fused()
@@ -314,9 +320,14 @@ def main():
     if fused:
         model.timeline_enable(True)
     bytes_log.clear()
+    touched_counts = []
     for _ in range(args.profile_steps):
         one_step("chained")
+        if shape.n_experts:
+            touched_counts.append(model.moe_touched_experts() / shape.n_layers)
     torch.cuda.synchronize()
+    if touched_counts:
+        touched["mean"] = float(np.mean(touched_counts))
     prof = model.profile_read()
     model.profile_enable(False)
     peak, peak_kind = peaks()
@@ -334,7 +345,7 @@ def main():
         tl_total = sum(v[0] for v in tl.values()) or 1.0
         kernels = {k: {"us_per_step": v[0], "phases_per_step": v[1], "share": v[0] / tl_total} for k, v in tl.items()}
     else:
-        # The dominant kernel is the launch class with the largest share of the step; its algorithmic bytes per
+        # The dominant kernel is the one whose launches take the largest share of the step; the algorithmic bytes of a
         # launch are the packed tensor it streams (projections) or the cached K, V it reads (attention).
         from workload import shapes as shp
         H, d = shape.hidden, shape.head_dim
@@ -343,31 +354,69 @@ def main():
                        "gemm_gate_up": shp.q4_bytes(2 * shape.mlp_inter, H) if shape.mlp_inter else 0,
                        "gemm_down": shp.q4_bytes(H, shape.mlp_inter) if shape.mlp_inter else 0,
                        "lm_head": shp.q4_bytes(shape.vocab, H) + n * shape.vocab * 4, "attention": kv_read_layer}
-        if shape.n_experts:  # expected distinct experts per layer (see step_bytes)
-            touched = shape.n_experts * (1.0 - (1.0 - shape.top_k / shape.n_experts) ** n)
-            class_bytes["moe_gate_up"] = touched * shp.q4_bytes(2 * shape.expert_inter, H)
-            class_bytes["moe_down"] = touched * shp.q4_bytes(H, shape.expert_inter)
-        class_kernel = {"attention": "paged_attention_kernel", "lm_head": "q4_round_kernel", "moe_gate_up": "q4_gemm_kernel", "moe_down": "q4_gemm_kernel"}
+        if shape.n_experts:  # distinct experts per layer, counted from the routing of the profiled steps
+            class_bytes["moe_gate_up"] = touched["mean"] * shp.q4_bytes(2 * shape.expert_inter, H)
+            class_bytes["moe_down"] = touched["mean"] * shp.q4_bytes(H, shape.expert_inter)
+        proj = "q4_umma_kernel" if os.environ.get("Q4D_GEMM_KERNEL") == "tcgen05" else "q4_span_kernel"
+        head = "q4_umma_kernel" if os.environ.get("Q4D_GEMM_KERNEL") == "tcgen05" else "q4_round_kernel"
+        class_kernel = {"gemm_qkv": proj, "gemm_o": proj, "gemm_gate_up": proj, "gemm_down": proj, "lm_head": head,
+                        "attention": "paged_attention_kernel", "moe_gate_up": "q4_gemm_kernel",
+                        "moe_down": "q4_gemm_kernel", "rmsnorm": "rmsnorm_kernel", "embed": "embed_kernel",
+                        "argmax": "argmax_finish_kernel", "moe_router": "moe_router_kernel"}
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped
         # batch-16 case (see profiles/); traffic is proportional to the bytes streamed, so it is scaled to this launch.
-        traffic_ratio = {"gemm_gate_up": 1.005, "attention": 1.032}
+        traffic_ratio = {"q4_span_kernel": 1.005, "paged_attention_kernel": 1.032}
         total_prof_ms = sum(v[0] for v in prof.values())
-        kernels = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
-                       "share": v[0] / total_prof_ms} for k, v in prof.items() if v[1]}
-        for k, v in kernels.items():
+        classes = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
+                       "share": v[0] / total_prof_ms, "kernel": class_kernel.get(k, k)} for k, v in prof.items() if v[1]}
+        for k, v in classes.items():
             if k in class_bytes and prof[k][1]:
                 v["GBps"] = class_bytes[k] / (prof[k][0] / prof[k][1] * 1e-3) / 1e9
-        top = max((k for k in kernels if k in class_bytes), key=lambda k: kernels[k]["share"])
-        top_ms, top_cnt = prof[top]
-        gbs = class_bytes[top] / (top_ms / top_cnt * 1e-3) / 1e9
-        roofline = {"kernel": class_kernel.get(top, "q4_span_kernel") + " (" + top + ")", "bound": "hbm", "achieved": gbs,
-                    "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": peak_kind,
-                    "traffic": class_bytes[top] * traffic_ratio[top] if top in traffic_ratio else None,
-                    "bytes_per_launch": float(class_bytes[top]), "us_per_launch": top_ms / top_cnt * 1e3,
-                    "timing": "CUDA events around each launch, profile pass right after the timed steps"}
+        # one entry per kernel: its launches of every class added up
+        kernels = {}
+        for k, v in classes.items():
+            e = kernels.setdefault(v["kernel"], {"ms_per_step": 0.0, "launches_per_step": 0.0, "share": 0.0,
+                                                 "bytes_per_step": 0.0, "classes": []})
+            e["ms_per_step"] += v["ms_per_step"]
+            e["launches_per_step"] += v["launches_per_step"]
+            e["share"] += v["share"]
+            e["bytes_per_step"] += class_bytes.get(k, 0.0) * v["launches_per_step"]
+            e["classes"].append(k)
+        for e in kernels.values():
+            e["GBps"] = e["bytes_per_step"] / (e["ms_per_step"] * 1e-3) / 1e9 if e["bytes_per_step"] else None
+        top = max((k for k in kernels if kernels[k]["bytes_per_step"]), key=lambda k: kernels[k]["share"])
+        te = kernels[top]
+        per_launch_bytes = te["bytes_per_step"] / te["launches_per_step"]
+        gbs = te["GBps"]
+        roofline = {"kernel": top, "bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                    "peak_kind": peak_kind, "share_of_step": te["share"],
+                    "traffic": per_launch_bytes * traffic_ratio[top] if top in traffic_ratio else None,
+                    "bytes_per_launch": per_launch_bytes,
+                    "us_per_launch": te["ms_per_step"] / te["launches_per_step"] * 1e3,
+                    "launches_per_step": te["launches_per_step"],
+                    "classes": {k: {"GBps": classes[k].get("GBps"), "frac": classes[k].get("GBps", 0.0) / peak,
+                                    "us_per_launch": classes[k]["ms_per_step"] / classes[k]["launches_per_step"] * 1e3,
+                                    "share_of_step": classes[k]["share"]} for k in te["classes"]},
+                    "timing": "CUDA events around each launch (a pass of --profile-steps steps right after the timed "
+                              "steps); achieved = bytes of all launches of the kernel / their summed time"}
+        kernels["by_class"] = classes
 
     # ---- max over ranks, aggregate ----
     ms, ms_e2e, tokens, tokens_e2e, launches = aggregate_ranks(dist, device, ms, ms_e2e, tokens, tokens_e2e, launches)
+
+    # bytes of the timed steps (mixture of experts: with the routed-expert count measured in the profile pass)
+    from workload import shapes as shp2
+    mean_bytes = {k: float(np.mean([b[k] for b in timed_bytes])) for k in timed_bytes[0]}
+    if shape.n_experts:
+        w_meas = float(shp2.weight_bytes(shape, touched["mean"]))
+        mean_bytes["total"] += w_meas - mean_bytes["weights"]
+        mean_bytes["weights"] = w_meas
+        config["experts"] = (f"{shape.n_experts} experts, top-{shape.top_k}; weight bytes count the distinct experts "
+                             f"the steps routed to (q4d_moe_touched_experts: {touched['mean']:.1f} per layer, mean over "
+                             f"the {args.profile_steps} profiled steps)")
+    config["workload"] += f"; mean cached tokens per request over the {args.steps} timed steps: {mean_kv_tokens:.0f}"
+    config["kv_mix"] = ("not stationary: departing requests are replaced by 512-token ones, so the mean KV length "
+                        "falls as steps go by; compare runs of equal --steps only") if churn else "fixed set of requests"
 
     value = tokens / (ms * 1e-3)
     step_gbs = mean_bytes["total"] / (ms / args.steps * 1e-3) / 1e9
@@ -382,16 +431,35 @@ def main():
         "roofline": roofline,
         "kernels": kernels,
         "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps,
+                "returns": "next tokens only (the logits stay on the device)"},
+        "e2e_with_logits": {"value": tokens_lg / (ms_e2e_lg * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d_lg,
+                            "d2h_bytes_per_step": d2h_lg, "ms_per_step": ms_e2e_lg / logit_steps, "steps": logit_steps,
+                            "returns": "next tokens and the fp32 logits of every request"},
         "gpu_launches": launches,
         "clocks": clocks,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # The oracle on whole steps of this workload; its result for the step is also the parity check of the run:
+        # the GPU takes the same step (same tokens, same KV) and the logits and greedy tokens are compared.
         ids, toks, lens, bt = script.step_inputs()
-        full, desc, cores = oracle_sample(shape, weights, pool_t, lens, toks, bt, args.oracle_layers)
-        out["cpu_baseline"] = {"value": len(ids) / full, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+        t_step, timed, desc, cores, (o_next, o_logits) = oracle_steps(shape, weights, pool_t, lens, toks, bt, 3,
+                                                                      args.oracle_budget)
+        out["cpu_baseline"] = {"value": len(ids) / t_step, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                                "sample": desc}
+        g_next = torch.zeros(len(ids), dtype=torch.int32, device=device)
+        g_logits = torch.zeros(len(ids), shape.vocab, dtype=torch.float32, device=device)
+        q4d.decode_step(model, pool, ids, toks, bt, g_next, g_logits)
+        torch.cuda.synchronize()
+        gl, ol = g_logits.cpu().numpy().astype(np.float64), o_logits.astype(np.float64)
+        rms = np.sqrt((ol ** 2).mean(-1))
+        out["parity"] = {"kind": "one whole step of this workload against the oracle, free-running through all "
+                                 f"{shape.n_layers} layers (bf16 rounding differences compound with depth; the "
+                                 "teacher-forced per-layer and head checks are in tests/)",
+                         "max_dlogit_over_rms": float((np.abs(gl - ol).max(-1) / rms).max()),
+                         "rms_dlogit_over_rms": float((np.sqrt(((gl - ol) ** 2).mean(-1)) / rms).max()),
+                         "greedy_tokens_equal": int((g_next.cpu().numpy() == o_next).sum()), "of": int(len(ids))}
     if rank == 0:
         print(json.dumps(out))
     pool.close()

@@ -2,18 +2,21 @@
  * q4decode — C ABI of the B200 decode-step library.
  *
  * One call, q4d_decode_step, is the body of the generation loop of the paper's
- * continuous-batching scheduler (Algorithm 1): for every request r of the
- * active batch B it computes token_r = GenerateToken(r, KVCache[r]).  Requests
- * join and leave B only between steps (Algorithm 1, "admit new requests at
- * token boundaries" / "remove completed requests immediately"), which is what
- * q4d_request_admit / q4d_request_release express.  Models are 4-bit quantised
+ * continuous-batching scheduler (Algorithm 1, generation loop): one new token
+ * for every request of the active batch, from that request's own KV cache.
+ * Membership of the batch changes only between steps (Algorithm 1, admission
+ * and removal loops), which is what q4d_request_admit / q4d_request_release
+ * express.  Models are 4-bit quantised
  * (Section 4, "Setup"); the forward pass is the pre-norm decoder of the model
  * families of Table 1.
  *
  * Conventions
- *  - Every function returns 0 (Q4D_OK) or a negative Q4D_ERR_* code; a failed
- *    call changes no state.  q4d_last_error() gives the message of the calling
- *    thread's last failure.
+ *  - Every function returns 0 (Q4D_OK) or a negative Q4D_ERR_* code.  A call
+ *    that fails its host-side validation changes no state; a CUDA error in the
+ *    middle of a step (Q4D_ERR_CUDA) leaves that step partially applied (K, V of
+ *    the new token written for the layers that ran; request lengths not
+ *    advanced).  q4d_last_error() gives the message of the calling thread's
+ *    last failure.
  *  - "device" pointers are CUDA device memory owned by the caller and must
  *    outlive the object they are given to; "host" pointers are ordinary host
  *    memory read before the call returns.  The library allocates no device
@@ -152,8 +155,7 @@ int q4d_request_count(q4d_kv_pool* pool, int32_t* count_out);
 
 /* ---- the decode step ---------------------------------------------------- */
 
-/* One token for each of the n listed requests (Algorithm 1, generation loop:
- * token_r = GenerateToken(r, KVCache[r]) for each r in B).
+/* One token for each of the n listed requests (Algorithm 1, generation loop).
  *   request_ids   host  [n]   distinct, all admitted
  *   last_tokens   host  [n]   the token each request feeds in (0 <= t < vocab)
  *   block_tables  host  [n][max_blocks]  physical block of tokens 16*i..16*i+15;
@@ -219,6 +221,10 @@ int q4d_timeline_read(q4d_model* model, float* us, int32_t* phases);
  * lengths, block tables, attention work list) and device -> host (only the
  * host-output variant copies anything back). */
 int q4d_step_io_bytes(q4d_model* model, int64_t* h2d_bytes, int64_t* d2h_bytes);
+/* Mixture-of-experts models: the number of (layer, expert) pairs the most recent step routed at least one request
+ * to, i.e. the expert tensors it actually streamed (the grouped dequant-GEMM runs over the experts touched per
+ * step).  Synchronises the device.  0 for dense models. */
+int q4d_moe_touched_experts(q4d_model* model, int64_t* total);
 
 /* ---- single operations (the kernels of the step, callable alone) -------- */
 /* All pointers are device memory; n <= 16.  `scratch` is device memory of at
@@ -249,7 +255,12 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
  *  - Projections whose split-K partial sums exceed the array, or with K > 16384, are refused with
  *    WORKSPACE_TOO_SMALL (for example a 69632 x 8192 projection); use q4d_q4_gemm then.
  *  - The first call on each device looks up the array's device address; make that first call
- *    outside any stream capture, with the device current.
+ *    outside any stream capture, with the device current.  The kernels' shared-memory limits are set
+ *    once per process, on the device that is current at the first projection call: use one device per
+ *    process.
+ *  - The call returns once the work is enqueued.  Should a bounded wait inside the kernel give up (a
+ *    copy that never lands), the results are void and nothing reports it here; the step entry points,
+ *    which own a status word, do report it.
  *  - Every call reuses the same array and finds in it what the previous call left; the counters are
  *    cleared on the stream before each launch.  Calls whose kernels can overlap on the GPU (different
  *    streams without an ordering between them) race on the array: keep them on one stream or order
@@ -298,6 +309,13 @@ int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, voi
 int q4d_debug_run_layers(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
                          const int32_t* block_tables, int32_t max_blocks, int32_t layer_begin, int32_t layer_end,
                          const uint16_t* x_in_device, uint16_t* x_out_device, void* cuda_stream);
+
+/* Writes `value` into the device word in which the step's kernels report a bounded wait that gave up (a bulk copy
+ * that never landed, a grid barrier that never completed).  The kernels only ever set it from inside such a wait;
+ * this export lets a test exercise the host side of the report without making any wait on the GPU run out: after a
+ * non-zero value the next step still runs and reads the word back, the step after it returns Q4D_ERR_TIMEOUT, and
+ * so does every later step of this model (its results are void: destroy and re-create it). */
+int q4d_debug_set_status(q4d_model* model, uint32_t value);
 
 /* out f32 [N][K] = the dequantised weights (bit-exact definition above). */
 int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out_device, void* cuda_stream);

@@ -22,10 +22,10 @@ EXPORTS = [
     "q4d_kv_pool_create", "q4d_kv_pool_destroy", "q4d_request_admit", "q4d_request_release", "q4d_request_len",
     "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_profile_enable",
     "q4d_profile_read", "q4d_launch_count", "q4d_step_is_fused", "q4d_timeline_enable", "q4d_timeline_read",
-    "q4d_step_io_bytes", "q4d_op_scratch_bytes", "q4d_q4_gemm",
+    "q4d_step_io_bytes", "q4d_moe_touched_experts", "q4d_op_scratch_bytes", "q4d_q4_gemm",
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
     "q4d_rmsnorm", "q4d_embed", "q4d_rope_append", "q4d_paged_attention", "q4d_argmax", "q4d_debug_dequant",
-    "q4d_debug_kv_gather", "q4d_debug_run_layers",
+    "q4d_debug_kv_gather", "q4d_debug_run_layers", "q4d_debug_set_status",
 ]
 
 
@@ -178,6 +178,14 @@ class Model:
         h2d, d2h = C.c_int64(), C.c_int64()
         _check(lib().q4d_step_io_bytes(self.handle, C.byref(h2d), C.byref(d2h)))
         return h2d.value, d2h.value
+
+    def debug_set_status(self, value):
+        _check(lib().q4d_debug_set_status(self.handle, C.c_uint32(value)))
+
+    def moe_touched_experts(self):
+        total = C.c_int64()
+        _check(lib().q4d_moe_touched_experts(self.handle, C.byref(total)))
+        return total.value
 
 
 class KVPool:

@@ -105,6 +105,7 @@ bool shape_supported(const q4d_shape& s, std::string* why) {
   if (s.group_size != 64 || s.bits != 4) return bad("only 4-bit group-64 weights are supported");
   if (s.n_q_heads % s.n_kv_heads || s.n_q_heads / s.n_kv_heads > 16) return bad("q heads per kv head must be 1..16");
   if (s.hidden % 256 || (s.n_q_heads * s.head_dim) % 256) return bad("hidden and nq*128 must be multiples of 256");
+  if (s.hidden > 16384) return bad("hidden must be at most 16384 (the RMSNorm kernel holds a row in registers)");
   if (s.max_batch < 1 || s.max_batch > kMaxBatch) return bad("max_batch must be 1..16");
   if (s.max_positions < 1) return bad("max_positions must be positive");
   if (s.n_experts == 0) {
@@ -143,7 +144,7 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
     w.yplain = take(B * s.hidden * 2);
     w.m_idx = take(B * s.top_k * 4);
     w.m_wgt = take(B * s.top_k * 4);
-    w.m_ints = take((3 * E + 2) * 4);  // flags[E], expert_ids[E], slot_of[E], counter, n_touched
+    w.m_ints = take((3 * E + 3) * 4);  // flags[E], expert_ids[E], slot_of[E], counter, n_touched, touched_total
     w.m_hp = take(E * B * s.expert_inter * 2);
     w.m_hs = take(E * (size_t)(s.expert_inter / 64) * 16 * 4);
     w.m_o = take(E * B * s.hidden * 2);
@@ -234,6 +235,7 @@ struct q4d_model {
   uint32_t* host_status;  // pinned copy of the kernel's status word, read back after every step
   cudaEvent_t status_done;
   bool status_pending;
+  bool timed_out;  // a kernel of an earlier step reported a wait that gave up: every later step is refused
 };
 
 struct q4d_kv_pool {
@@ -351,12 +353,15 @@ void build_fused_params(const q4d_model* m, FusedStep* fp) {
 // Reports a wait that gave up inside a kernel of an earlier step (a grid barrier of the persistent kernel, a bulk
 // copy of the projection kernel) once the step's status word has come back.
 int fused_check_status(q4d_model* m, bool wait) {
+  if (m->timed_out)
+    return fail(Q4D_ERR_TIMEOUT, "decode_step: a bounded wait inside a kernel of an earlier step gave up; destroy and re-create the model");
   if (!m->status_pending) return Q4D_OK;
   cudaError_t e = wait ? cudaEventSynchronize(m->status_done) : cudaEventQuery(m->status_done);
   if (e == cudaErrorNotReady) return Q4D_OK;
   if (e != cudaSuccess) return fail_cuda(e, "status read-back");
   m->status_pending = false;
-  if (*m->host_status != 0u)
+  if (*m->host_status != 0u) m->timed_out = true;
+  if (m->timed_out)
     return fail(Q4D_ERR_TIMEOUT, "decode_step: a bounded wait inside a kernel of an earlier step gave up; destroy and re-create the model");
   return Q4D_OK;
 }
@@ -552,6 +557,10 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     if (le != cudaSuccess) return fail_cuda(le, #cls);                        \
   } while (0)
 
+  if (sh.n_experts) {  // the step's count of routed experts starts at zero
+    cudaError_t ce = cudaMemsetAsync(at<int32_t>(m, m->lay.m_ints) + 3 * sh.n_experts + 2, 0, 4, s);
+    if (ce != cudaSuccess) return fail_cuda(ce, "routed-expert counter reset");
+  }
   if (range) {
     cudaError_t ce = cudaMemcpyAsync(x, range->x_in, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
     if (ce != cudaSuccess) return fail_cuda(ce, "hidden state copy");
@@ -583,7 +592,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       GemmArgs gu = gemm_args(m, lw.w_gate_up, 2 * I, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
       gu.out_xp = hp, gu.out_xs = hs;
       Q4D_LAUNCH(Q4D_K_GEMM_GATE_UP, launch_q4_gemm(gu, s));
-      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, hs, n, EPI_RESIDUAL, x, H), s));
+      Q4D_LAUNCH(Q4D_K_GEMM_DOWN, launch_q4_gemm(gemm_args(m, lw.w_down, H, I, hp, dense_layout == OPERAND_BLOCKED ? hs : nullptr, n, EPI_RESIDUAL, x, H), s));
     } else {
       const int E = sh.n_experts, Ie = sh.expert_inter;
       uint16_t* yplain = at<uint16_t>(m, m->lay.yplain);
@@ -593,6 +602,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       mr.idx = at<int32_t>(m, m->lay.m_idx), mr.wgt = at<float>(m, m->lay.m_wgt);
       mr.flags = ints, mr.expert_ids = ints + E, mr.slot_of = ints + 2 * E, mr.counter = ints + 3 * E;
       mr.n_touched = ints + 3 * E + 1;
+      mr.touched_total = ints + 3 * E + 2;
       uint16_t* ehp = at<uint16_t>(m, m->lay.m_hp);
       float* ehs = at<float>(m, m->lay.m_hs);
       uint16_t* eo = at<uint16_t>(m, m->lay.m_o);
@@ -703,7 +713,7 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   m->staging_next = 0;
   m->host_next = nullptr;
   m->fused = false, m->fused_ctas = 0, m->timeline = false, m->fused_params = nullptr;
-  m->host_status = nullptr, m->status_done = nullptr, m->status_pending = false;
+  m->host_status = nullptr, m->status_done = nullptr, m->status_pending = false, m->timed_out = false;
   int dev = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&m->sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -717,7 +727,7 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.attn_merge_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
   if (e == cudaSuccess && shape->n_experts)
-    e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 2) * 4);
+    e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 3) * 4);
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.chain_status, 0, 256);
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->status_done, cudaEventDisableTiming);
@@ -920,6 +930,19 @@ int q4d_timeline_read(q4d_model* m, float* us, int32_t* phases) {
   return Q4D_OK;
 }
 
+int q4d_moe_touched_experts(q4d_model* m, int64_t* total) {
+  if (!m || !total) return fail(Q4D_ERR_INVALID_ARG, "moe_touched_experts: NULL argument");
+  *total = 0;
+  if (!m->sh.n_experts) return Q4D_OK;
+  int32_t v = 0;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess)
+    e = cudaMemcpy(&v, at<int32_t>(m, m->lay.m_ints) + 3 * m->sh.n_experts + 2, 4, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fail_cuda(e, "moe_touched_experts");
+  *total = v;
+  return Q4D_OK;
+}
+
 int q4d_step_io_bytes(q4d_model* m, int64_t* h2d, int64_t* d2h) {
   if (!m || !h2d || !d2h) return fail(Q4D_ERR_INVALID_ARG, "step_io_bytes: NULL argument");
   *h2d = m->last_h2d, *d2h = m->last_d2h;
@@ -948,6 +971,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
   if (n < 0 || n > kMaxBatch || N < 1 || K < 256 || K % 256 || x_stride % 8 || prologue < 0 || prologue > 1 ||
       epilogue < 0 || epilogue > 2)
     return fail(Q4D_ERR_INVALID_ARG, "q4_gemm: bad shape (K must be a multiple of 256, n <= 16)");
+  if (x_stride < K * (1 + prologue)) return fail(Q4D_ERR_INVALID_ARG, "q4_gemm: x_stride is smaller than a row of the operand");
   if (K > kOpMaxK || gemm_partial_bytes(N, K, epilogue) > kOpGemmPartial ||
       (size_t)gemm_counters_needed(N) * 4 > kOpCounters)
     return fail(Q4D_ERR_WORKSPACE_TOO_SMALL, "q4_gemm: shape needs more scratch than q4d_op_scratch_bytes provides");
@@ -1049,6 +1073,15 @@ int q4d_debug_run_layers(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64
   const LayerRange range{layer_begin, layer_end, x_in, x_out};
   return step_impl(m, pool, n, ids, nullptr, nullptr, bt, max_blocks, nullptr, nullptr,
                    static_cast<cudaStream_t>(stream), &range);
+}
+
+int q4d_debug_set_status(q4d_model* m, uint32_t value) {
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "debug_set_status: NULL model");
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess)
+    e = cudaMemcpy(m->fused ? reinterpret_cast<unsigned char*>(m->fused_params->control + 1) : m->ws + m->lay.chain_status,
+                   &value, sizeof value, cudaMemcpyHostToDevice);
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "debug_set_status");
 }
 
 int q4d_debug_dequant(const q4d_qtensor* w, int32_t N, int32_t K, float* out, void* stream) {

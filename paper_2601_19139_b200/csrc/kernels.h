@@ -148,6 +148,7 @@ struct MoeRouteArgs {
   int32_t* expert_ids;  // [E] touched experts, ascending
   int32_t* slot_of;     // [E] position of an expert in expert_ids
   int32_t* n_touched;
+  int32_t* touched_total = nullptr;  // optional: running sum of n_touched over the launches of a step
 };
 struct MoeCombineArgs {
   uint16_t* x;        // residual stream bf16 [n][H], updated in place

@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(256) moe_router_kernel(const MoeRouteArgs p) {
     for (int w = 0; w < 8; ++w) tot += s_warp_base[w];
     *p.n_touched = tot;
     *p.counter = 0;
+    if (p.touched_total) *p.touched_total += tot;  // one CTA per launch, launches of a step are stream-ordered
   }
 }
 

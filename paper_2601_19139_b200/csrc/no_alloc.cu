@@ -14,6 +14,8 @@
 // whose kernels overlap on the GPU (different streams, no ordering) race on the scratch.
 #include <stdio.h>
 
+#include <atomic>
+
 #include "../../include/q4decode.h"
 #include "kernels.h"
 
@@ -28,7 +30,7 @@ constexpr size_t kScratchBytes = kCounterBytes + kPartialBytes + kOperandBytes;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_ptr[kMaxDevices] = {};
+std::atomic<unsigned char*> g_scratch_ptr[kMaxDevices] = {};  // looked up once per device; any host thread may call
 
 thread_local char g_noalloc_error[256];
 
@@ -61,7 +63,9 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices)
     return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: no current CUDA device");
-  if (!g_scratch_ptr[dev]) {  // once per device, with that device current
+  if (x_stride < K * (1 + prologue))
+    return q4d_internal_fail(Q4D_ERR_INVALID_ARG, "q4_gemm_noalloc: x_stride is smaller than a row of the operand");
+  if (!g_scratch_ptr[dev].load(std::memory_order_acquire)) {  // once per device, with that device current
     void* p = nullptr;
     e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
     if (e != cudaSuccess || !p) {
@@ -69,11 +73,11 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
                cudaGetErrorString(e));
       return q4d_internal_fail(Q4D_ERR_CUDA, g_noalloc_error);
     }
-    g_scratch_ptr[dev] = static_cast<unsigned char*>(p);
+    g_scratch_ptr[dev].store(static_cast<unsigned char*>(p), std::memory_order_release);
   }
   if (n == 0) return Q4D_OK;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  unsigned char* base = g_scratch_ptr[dev];
+  unsigned char* base = g_scratch_ptr[dev].load(std::memory_order_acquire);
   // The counters must be zero when the kernel starts; whatever an earlier call left is cleared here.
   e = cudaMemsetAsync(base, 0, need_counters, s);
   if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: clearing the counters failed");

@@ -76,7 +76,7 @@ def _run_steps(q4d, sc, steps):
     logits = torch.zeros(n, shape.vocab, dtype=torch.float32, device="cuda")
     agree = total = 0
     worst_max = worst_rms = 0.0
-    sc.per_request_max = []
+    sc.per_request_max, sc.per_request_rms = [], []
     toks = sc.tokens.copy()
     for _ in range(steps):
         bt = sc.block_tables()
@@ -86,15 +86,20 @@ def _run_steps(q4d, sc, steps):
         emax, erms = _logit_err(logits.cpu().numpy(), o_logits)
         worst_max, worst_rms = max(worst_max, float(emax.max())), max(worst_rms, float(erms.max()))
         sc.per_request_max.extend(float(v) for v in emax)
+        sc.per_request_rms.extend(float(v) for v in erms)
         agree += int((nxt.cpu().numpy() == o_next).sum())
         total += n
         for r in range(n):
             blk, slot = bt[r, sc.lens[r] // 16], sc.lens[r] % 16
             # layer 0 sees identical inputs on both sides: its appended K, V match up to rounding.  A QKV output that
             # rounds one bf16 step apart (fp32 vs fp64 sums) moves, through the rotation k'_i = k_i c - k_(i+64) s, a
-            # small k'_i by one step of the larger partner: a few steps of k'_i, on a small fraction of elements.
+            # small k'_i by one step of the larger partner: a few steps of k'_i.  And when a single element of the
+            # normed input rounds differently (fp32 vs fp64 sum of squares), every output of the projection moves by
+            # about 2^-9 / sqrt(H) of its size and a few per cent of them cross a rounding boundary (measured: up to
+            # 12 % of a request's K and V elements one step apart, all heads alike).  A misplaced append (wrong slot,
+            # head or rotation) differs in every element and by far more than eight steps.
             assert_bf16_close(bits(sc.pool[0, :, blk, :, slot]), sc.host_pool[0, :, blk, :, slot], max_ulp=8,
-                              max_mismatch_frac=0.03, what="layer-0 appended kv")
+                              max_mismatch_frac=0.25, what="layer-0 appended kv")
             sc.pool[:, :, blk, :, slot] = from_bits(sc.host_pool[:, :, blk, :, slot])
             assert pool.request_len(int(ids[r])) == sc.lens[r] + 1
             sc.lens[r] += 1
@@ -229,6 +234,32 @@ def test_qwen3_0p6b_layers_and_head_teacher_forced(q4d):
     assert agree / total >= 0.995, (agree, total)
 
 
+def test_qwen3_8b_widths_layers_and_head_teacher_forced(q4d):
+    """The benchmarked widths (hidden 4096, 32 query / 8 kv heads, MLP 12288: the down projection's K is cut in
+    parts), two layers deep, 16 requests with lengths drawn log-uniformly from [256, 8192] and one of them beyond
+    8192 tokens: each layer through the step's own launch sequence from the oracle's input, then the head."""
+    import dataclasses
+    shape = dataclasses.replace(shapes.QWEN3_8B, name="qwen3-8b-shaped-2layers", n_layers=2)
+    rng = np.random.default_rng(3)
+    lens = gen.draw_lengths(16, 256, 8192, rng, True).tolist()
+    lens[5] = 8300
+    sc = Scenario(shape, lens, seed=11)
+    _, emax, same, n = _layerwise(q4d, sc)
+    assert emax <= LOGIT_TOL and same == n
+
+
+def test_llama32_3b_widths_layers_and_head_teacher_forced(q4d):
+    """The Llama-3.2-3B widths (hidden 3072, 24 query / 8 kv heads: three query heads per kv head, no qk-norm,
+    eps 1e-5, tied embedding and head), two layers deep, 16 requests with lengths uniform in [512, 4096]."""
+    import dataclasses
+    shape = dataclasses.replace(shapes.LLAMA32_3B, name="llama-3.2-3b-shaped-2layers", n_layers=2)
+    rng = np.random.default_rng(4)
+    lens = gen.draw_lengths(16, 512, 4096, rng).tolist()
+    sc = Scenario(shape, lens, seed=12)
+    _, emax, same, n = _layerwise(q4d, sc)
+    assert emax <= LOGIT_TOL and same == n
+
+
 def test_moe_30b_shape_layers_and_head_teacher_forced(q4d):
     """The MoE-30B layer at full width (128 experts, 8 per token, 768-wide experts, hidden 2048) and the full
     vocabulary head, two layers deep, 16 requests: each layer from the oracle's input."""
@@ -269,21 +300,182 @@ def test_qwen3_0p6b_batch16_whole_steps(q4d):
 
 
 def _check_against_drift_band(q4d, sc, steps):
-    """Whole-step logits may drift from the oracle by what bf16 rounding chaos allows.  The yardstick is the oracle
-    against itself with fp32 instead of fp64 accumulation in the projections (nothing else changed) on the same
-    inputs: the GPU's rms logit error must stay within 3x of that drift (and the max within 3x of its max)."""
+    """Whole-step logits may drift from the oracle by what bf16 rounding chaos allows.  The yardstick is a second
+    build of the oracle's source whose projections accumulate in fp32 instead of fp64 (tests/fp32_probe.py; nothing
+    else differs) on the same inputs: a correct fp32 implementation can be no closer to the definition than that.
+    The GPU's rms logit error must stay within 1.5x of that variant's, its largest error within 2x of its largest.
+    Returns the figures for the report."""
     bt = sc.block_tables()
     ref = sc.oracle.decode_step(sc.host_pool.copy(), 16, sc.lens, sc.tokens, bt)
     with fp32_probe.fp32_accumulation():
         probe = sc.oracle.decode_step(sc.host_pool.copy(), 16, sc.lens, sc.tokens, bt)
     pmax, prms = _logit_err(probe[1], ref[1])
-    band_max, band_rms = float(pmax.max()), float(prms.max())
+    band_max, band_rms = float(pmax.max()), float(np.sqrt((prms ** 2).mean()))
     agree, total, worst_max, worst_rms = _run_steps(q4d, sc, steps)
-    print(f"[{sc.shape.name}] oracle fp32-accumulate drift: max {band_max:.3e} rms {band_rms:.3e}, "
-          f"tokens equal {(probe[0] == ref[0]).sum()}/{len(sc.lens)}")
-    rms_b, max_b = drift_bounds(sc.shape.n_layers)
-    assert worst_rms <= min(max(3.0 * band_rms, 2e-3), rms_b), (worst_rms, band_rms, rms_b)
-    assert worst_max <= min(max(3.0 * band_max, LOGIT_TOL), max_b), (worst_max, band_max, max_b)
+    print(f"[{sc.shape.name}] fp32-accumulating oracle variant vs oracle: max {band_max:.3e} rms {band_rms:.3e}, "
+          f"tokens equal {(probe[0] == ref[0]).sum()}/{len(sc.lens)}; GPU vs oracle: max {worst_max:.3e} "
+          f"rms {worst_rms:.3e}, tokens equal {agree}/{total}")
+    assert worst_rms <= max(1.5 * float(prms.max()), 2e-3), (worst_rms, float(prms.max()))
+    assert worst_max <= max(2.0 * band_max, LOGIT_TOL), (worst_max, band_max)
+    gpu_rms = float(np.sqrt(np.mean(np.square(sc.per_request_rms))))   # over requests (and steps), like band_rms
+    return band_max, band_rms, worst_max, gpu_rms, agree, total
+
+
+def test_qwen3_0p6b_drift_over_five_seeds(q4d):
+    """Full depth (28 layers), batch 16, one free-running step for each of five independent models and batches:
+    the GPU's distance from the oracle against the fp32-accumulating variant's, seed by seed.  The table this prints
+    is the measured answer to what the logit tolerance can mean at full depth."""
+    rng = np.random.default_rng(0)
+    lens = gen.draw_lengths(16, 128, 2048, rng).tolist()
+    rows = []
+    for seed in (21, 22, 23, 24, 25):
+        sc = Scenario(shapes.QWEN3_0P6B, lens, seed=seed)
+        rows.append(_check_against_drift_band(q4d, sc, steps=1))
+        del sc
+        torch.cuda.empty_cache()
+    g_rms, p_rms = np.mean([r[3] for r in rows]), np.mean([r[1] for r in rows])
+    agree, total = sum(r[4] for r in rows), sum(r[5] for r in rows)
+    print(f"[drift over 5 seeds] GPU rms {g_rms:.3e} vs fp32 variant rms {p_rms:.3e} (ratio {g_rms / p_rms:.2f}); "
+          f"GPU greedy tokens equal to the oracle's on {agree}/{total} free-running decisions")
+    assert g_rms <= 1.5 * p_rms
+
+
+def test_qwen3_0p6b_churn_64_steps_token_agreement(q4d, step_kernel):
+    """The 0.6B shape, 16 requests, 64 steps with requests leaving and joining every 8 steps (teacher-forced between
+    steps: both sides start every step from the same tokens and the same KV): 1024 greedy decisions, each taken
+    free-running through 28 layers.  Reported: agreement with the oracle.  Asserted: the agreement stays above 90 %
+    (the fp32-accumulating variant of the oracle itself agrees with the oracle on about 90-95 % of such decisions),
+    every logit vector stays inside the drift band, and every disagreement is a near-tie of the oracle's logits."""
+    if step_kernel == "fused":
+        pytest.skip("long run: once, with the default step path")
+    shape = shapes.QWEN3_0P6B
+    rng = np.random.default_rng(7)
+    lens = gen.draw_lengths(16, 128, 2048, rng).tolist()
+    sc = Scenario(shape, lens + [512] * 28, seed=31, extra_blocks=64)     # 28 more requests wait to be admitted
+    model = q4d.Model(shape, sc.weights)
+    pool = q4d.KVPool(model, sc.pool)
+    active = list(range(16))
+    waiting = list(range(16, 44))
+    for r in active:
+        pool.request_admit(r, sc.lens[r])
+    toks = {r: int(sc.tokens[r]) for r in range(44)}
+    nxt = torch.zeros(16, dtype=torch.int32, device="cuda")
+    lg = torch.zeros(16, shape.vocab, dtype=torch.float32, device="cuda")
+    agree = total = 0
+    worst = 0.0
+    rms_b, max_b = drift_bounds(shape.n_layers)
+    for step in range(64):
+        if step and step % 8 == 0:          # membership changes at a token boundary (Algorithm 1)
+            for r in [active[i] for i in sorted(rng.choice(16, size=3, replace=False))]:
+                pool.request_release(r)
+                active.remove(r)
+            for _ in range(3):
+                r = waiting.pop(0)
+                pool.request_admit(r, sc.lens[r])
+                active.append(r)
+        bt = sc.block_tables()
+        rows = list(active)
+        q4d.decode_step(model, pool, np.array(rows, dtype=np.int64), np.array([toks[r] for r in rows], dtype=np.int32),
+                        bt[rows], nxt, lg)
+        torch.cuda.synchronize()
+        o_next, o_logits, _ = sc.oracle.decode_step(sc.host_pool, 16, [sc.lens[r] for r in rows],
+                                                    [toks[r] for r in rows], bt[rows])
+        g = lg.cpu().numpy()
+        emax, _ = _logit_err(g, o_logits)
+        worst = max(worst, float(emax.max()))
+        g_next = nxt.cpu().numpy()
+        for i, r in enumerate(rows):
+            total += 1
+            if g_next[i] == o_next[i]:
+                agree += 1
+            else:   # the GPU's choice must be within reach of the oracle's best logit given the logit error
+                o = o_logits[i].astype(np.float64)
+                rms = np.sqrt((o ** 2).mean())
+                assert o[o_next[i]] - o[g_next[i]] <= 2.0 * emax[i] * rms + 1e-12
+            blk, slot = bt[r, sc.lens[r] // 16], sc.lens[r] % 16
+            sc.pool[:, :, blk, :, slot] = from_bits(sc.host_pool[:, :, blk, :, slot])
+            sc.lens[r] += 1
+            toks[r] = int(o_next[i])
+    pool.close()
+    model.close()
+    print(f"[{shape.name}] churn, 64 steps: greedy tokens equal on {agree}/{total} = {agree / total:.2%}; "
+          f"largest |dlogit|/rms {worst:.3e}")
+    assert worst <= max_b
+    assert agree / total >= 0.90
+
+
+def test_requests_sharing_prefix_blocks(q4d):
+    """Two requests list the same physical blocks for a shared 48-token prefix (read-only) and own their later
+    blocks; a third shares nothing.  The results must be bit-identical to those of the same batch with the prefix
+    stored twice, stay close to the oracle's, and the shared blocks must come out unchanged."""
+    shape = shapes.toy("gpu-toy-shared-prefix", hidden=512, n_q_heads=8, n_kv_heads=2, mlp_inter=768, vocab=2000)
+    sc = Scenario(shape, [70, 55, 33], seed=13, extra_blocks=16)
+    own = list(sc.blocks[1][:3])
+    shared = list(sc.blocks[0][:3])
+    sc.pool[:, :, own] = sc.pool[:, :, shared]          # request 1 has the same first 48 tokens as request 0
+    saved = sc.pool.clone()
+    model = q4d.Model(shape, sc.weights)
+    ids = np.arange(3, dtype=np.int64)
+
+    def run(share):
+        sc.pool.copy_(saved)
+        sc.blocks[1][:3] = shared if share else own
+        pool = q4d.KVPool(model, sc.pool)
+        for r in range(3):
+            pool.request_admit(r, sc.lens[r])
+        nxt = torch.zeros(3, dtype=torch.int32, device="cuda")
+        lg = torch.zeros(3, shape.vocab, dtype=torch.float32, device="cuda")
+        bt = sc.block_tables()
+        assert (list(bt[0, :3]) == list(bt[1, :3])) == share and bt[0, 3] != bt[1, 3]
+        q4d.decode_step(model, pool, ids, sc.tokens, bt, nxt, lg)
+        torch.cuda.synchronize()
+        pool.close()
+        return nxt.clone(), lg.clone(), bt
+
+    n_sep, lg_sep, _ = run(False)
+    n_sh, lg_sh, bt = run(True)
+    assert torch.equal(lg_sh, lg_sep) and torch.equal(n_sh, n_sep)
+    assert torch.equal(sc.pool[:, :, shared], saved[:, :, shared])           # the shared blocks were only read
+    host_pool = orc.to_np(saved).copy()
+    o_next, o_logits, _ = sc.oracle.decode_step(host_pool, 16, sc.lens, sc.tokens, bt)
+    emax, _ = _logit_err(lg_sh.cpu().numpy(), o_logits)
+    assert emax.max() <= 2 * LOGIT_TOL, emax      # two layers, free-running: rounding differences only
+    model.close()
+
+
+def test_timeout_report_reaches_the_caller(q4d):
+    """The host side of Q4D_ERR_TIMEOUT: the kernels set a status word when a bounded wait gives up.  Here the word
+    is set from the host (no wait on the GPU is made to run out): the step after the next one is refused with -10,
+    so is every later one, and a re-created model works again."""
+    shape = shapes.toy("gpu-toy-timeout", hidden=256, n_q_heads=4, n_kv_heads=2, mlp_inter=512, vocab=1024)
+    sc = Scenario(shape, [10, 20], seed=14)
+    model = q4d.Model(shape, sc.weights)
+    pool = q4d.KVPool(model, sc.pool)
+    ids = np.array([1, 2], dtype=np.int64)
+    pool.request_admit(1, 10)
+    pool.request_admit(2, 20)
+    nxt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    bt = sc.block_tables()
+    q4d.decode_step(model, pool, ids, sc.tokens, bt, nxt)        # a healthy step
+    torch.cuda.synchronize()
+    model.debug_set_status(3)
+    q4d.decode_step(model, pool, ids, sc.tokens, bt, nxt)        # runs, and reads the word back
+    torch.cuda.synchronize()
+    for _ in range(2):
+        with pytest.raises(q4d.Q4dError) as ei:
+            q4d.decode_step(model, pool, ids, sc.tokens, bt, nxt)
+        assert ei.value.code == -10
+    assert pool.request_len(1) == 12                              # the refused steps changed nothing
+    pool.close()
+    model.close()
+    model = q4d.Model(shape, sc.weights)                          # the workspace is reinitialised
+    pool = q4d.KVPool(model, sc.pool)
+    pool.request_admit(1, 12)
+    pool.request_admit(2, 22)
+    q4d.decode_step(model, pool, ids, sc.tokens, sc.block_tables(), nxt)
+    torch.cuda.synchronize()
+    pool.close()
+    model.close()
 
 
 def test_batch_invariance_and_determinism(q4d):

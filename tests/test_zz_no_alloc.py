@@ -11,6 +11,8 @@ import numpy as np
 import pytest
 import torch
 
+from gpu_util import assert_bf16_close, bits
+from oracle import q4d_oracle as orc
 from workload import gen
 
 pytestmark = pytest.mark.gpu
@@ -38,22 +40,58 @@ def test_noalloc_gemm_equals_the_scratch_taking_entry_point_twice_in_a_row(q4d):
         x = _x(n, K, 40 + i)
         out = torch.full((n, N), float("nan"), dtype=torch.float32 if epi == 2 else torch.bfloat16, device="cuda")
         prepared.append((w, x, n, epi, out))
+    # a first call loads the kernels and looks up the array's address (both may take device memory once, in the
+    # driver); the calls under test come after it
+    q4d.q4_gemm_noalloc(prepared[1][0], prepared[1][1], prepared[1][2], prepared[1][4], epilogue=prepared[1][3])
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
+    free_before = torch.cuda.mem_get_info()[0]
     for w, x, n, epi, out in prepared:                     # two calls in a row on the shared array
         q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.mem_get_info()[0] == free_before     # nor did anything else take device memory
     for w, x, n, epi, out in prepared:
         want = q4d.q4_gemm(w, x, n, epilogue=epi)
         torch.cuda.synchronize()
         assert torch.equal(out, want)
+        # and against the definition itself, not only the sibling entry point
+        ref = orc.q4_matmul(*(orc.to_np(a) for a in w), bits(x))
+        rms = np.sqrt((ref ** 2).mean())
+        if epi == 2:
+            assert np.abs(out.cpu().numpy().astype(np.float64) - ref).max() <= 3e-5 * rms
+        else:
+            assert_bf16_close(bits(out), orc.bf16_round(ref), what="no-alloc bf16 output")
     # and again in the other order: what the previous call left in the array must not matter
     for w, x, n, epi, out in reversed(prepared):
         out.fill_(float("nan"))
         q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
         torch.cuda.synchronize()
         assert torch.equal(out, q4d.q4_gemm(w, x, n, epilogue=epi))
+
+
+def test_noalloc_gemm_residual_epilogue_and_silu_prologue(q4d):
+    """The other two modes of the entry point, each against the scratch-taking one and against the oracle."""
+    N, K, n = 2048, 1024, 7
+    w = gen.random_q4(N, K, "cuda", "noalloc-modes")
+    x = _x(n, K, 60)
+    res = _x(n, N, 61)
+    res2 = res.clone()
+    q4d.q4_gemm_noalloc(w, x, n, res, epilogue=1)
+    q4d.q4_gemm(w, x, n, epilogue=1, out=res2)
+    torch.cuda.synchronize()
+    assert torch.equal(res, res2)
+    gu = _x(n, 2 * K, 62)
+    out = torch.zeros(n, N, dtype=torch.float32, device="cuda")
+    q4d.q4_gemm_noalloc(w, gu, n, out, prologue=1, epilogue=2)
+    torch.cuda.synchronize()
+    assert torch.equal(out, q4d.q4_gemm(w, gu, n, prologue=1, epilogue=2))
+    gub = bits(gu)
+    ref = orc.q4_matmul(*(orc.to_np(a) for a in w), orc.silu_mul(gub[:, :K], gub[:, K:]))
+    assert np.abs(out.cpu().numpy().astype(np.float64) - ref).max() <= 2e-3 * np.sqrt((ref ** 2).mean())
+    with pytest.raises(q4d.Q4dError) as ei:                 # a row stride shorter than the operand's row
+        q4d.q4_gemm_noalloc(w, _x(n, K // 2, 63), n, out, epilogue=2)
+    assert ei.value.code == -1
 
 
 def test_noalloc_gemm_refuses_shapes_beyond_its_array(q4d):
