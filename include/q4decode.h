@@ -172,6 +172,29 @@ int q4d_decode_step(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_
                     const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
                     int32_t* next_tokens, float* logits, void* cuda_stream);
 
+/* Per-request sampling settings of one step (host arrays of n entries each, read before the call returns).  The
+ * paper's scheduler only says that a token is generated per request (Algorithm 1, generation loop) and is silent on
+ * how it is chosen; this is the usual temperature / top-k / top-p rule with the random draw supplied by the caller,
+ * so that a run is reproducible from its seed:
+ *   temperature <= 0 : the greedy token (largest logit, lowest index among equals); the other fields are ignored
+ *   otherwise        : integer weights w_j = rint(2^40 exp((l_j - max l) / temperature));
+ *                      top_k in 1..vocab-1 keeps the tokens whose logit is >= the k-th largest (ties at the cut
+ *                      stay), any other value keeps all; top_p < 1 then keeps { l_j >= c } for the largest c whose
+ *                      set holds at least ceil(top_p * kept weight); with W the weight kept and t = floor(u * W)
+ *                      (u in [0, 1)), the tokens are walked by descending logit, ascending index among equal
+ *                      logits, and the first whose running weight exceeds t is the result. */
+typedef struct {
+  const float* temperature;
+  const int32_t* top_k;
+  const float* top_p;
+  const float* u;
+} q4d_sampling;
+
+/* q4d_decode_step whose next_tokens are drawn by the rule above from the step's logits instead of the argmax. */
+int q4d_decode_step_sampled(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_t* request_ids,
+                            const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
+                            const q4d_sampling* sampling, int32_t* next_tokens, float* logits, void* cuda_stream);
+
 /* Same step, but the fed-in tokens are read from device memory when the
  * kernels run (e.g. the next_tokens buffer of the previous step), so a loop
  * of steps needs no host round trip.  Token values are then not validated on
@@ -296,6 +319,10 @@ int q4d_paged_attention(const uint16_t* q, const uint16_t* pool_layer_k, const u
                         const int32_t* lens_device, const int32_t* block_tables_device,
                         int32_t max_blocks, int32_t chunk_tokens /* 0 = auto */, uint16_t* out,
                         void* scratch, void* cuda_stream);
+
+/* next[r] drawn from logits f32 [n][vocab] (device) by the rule of q4d_sampling (host arrays). */
+int q4d_sample(const float* logits, int32_t n, int32_t vocab, const q4d_sampling* sampling, int32_t* next,
+               void* cuda_stream);
 
 /* next[r] = argmax_j logits[r][j], lowest index on ties. */
 int q4d_argmax(const float* logits, int32_t n, int32_t vocab, int32_t* next, void* cuda_stream);

@@ -280,3 +280,45 @@ class OracleModel:
         if rc != 0:
             raise RuntimeError(f"orc_decode_step failed: {rc}")
         return nxt, logits, taps
+
+
+# ------------------------------------------------------------------ sampling
+# The paper's scheduler generates "a token" per request (Algorithm 1, generation loop) and says nothing about how
+# it is chosen.  The reading built here is the usual temperature / top-k / top-p rule with the random draw u given by
+# the caller, written out plainly (a sort, a running sum) in fp64 with integer weights:
+#   w_j = rint(2^40 exp((l_j - max l) / T));  top-k keeps logits >= the k-th largest (ties at the cut stay);
+#   top-p keeps logits >= c for the largest c whose set weighs >= ceil(top_p * kept weight);
+#   t = floor(u * W) over the kept weight W; walk by (descending logit, ascending index); first running weight > t.
+
+def sampling_table(logits, temperature, top_k, top_p):
+    """(order, weights in that order, number of kept tokens): `order` lists all token ids by descending logit and
+    ascending index among equal logits; the first `kept` of them survive top-k and top-p."""
+    l = np.asarray(logits, dtype=np.float64)
+    V = l.size
+    order = np.lexsort((np.arange(V), -l))
+    ls = l[order]
+    w = np.rint(np.exp((ls - ls[0]) / float(temperature)) * 2.0 ** 40).astype(np.int64)
+    kept = V
+    if 0 < top_k < V:
+        kth = ls[top_k - 1]
+        kept = int(np.searchsorted(-ls, -kth, side="right"))          # every logit >= the k-th largest
+    if top_p < 1.0:
+        Wk = int(w[:kept].sum())
+        target = min(max(int(np.ceil(float(np.float32(top_p)) * float(Wk))), 1), Wk)
+        cum = np.cumsum(w[:kept])
+        first = int(np.searchsorted(cum, target, side="left"))         # first position whose running weight >= target
+        c = ls[first]
+        kept = min(kept, int(np.searchsorted(-ls, -c, side="right")))  # and every token tied with it
+    return order, w, kept
+
+
+def sample_token(logits, temperature, top_k, top_p, u):
+    """The token the rule draws for one request."""
+    l = np.asarray(logits, dtype=np.float64)
+    if not temperature > 0.0:
+        return int(np.flatnonzero(l == l.max())[0])
+    order, w, kept = sampling_table(l, temperature, top_k, top_p)
+    W = int(w[:kept].sum())
+    t = min(int(float(np.float32(u)) * float(W)), W - 1)
+    cum = np.cumsum(w[:kept])
+    return int(order[int(np.searchsorted(cum, t, side="right"))])      # first running weight > t

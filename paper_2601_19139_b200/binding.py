@@ -20,7 +20,7 @@ K_NAMES = ["embed", "rmsnorm", "gemm_qkv", "rope_append", "attention", "attn_mer
 EXPORTS = [
     "q4d_last_error", "q4d_model_workspace_bytes", "q4d_model_create", "q4d_model_destroy", "q4d_kv_pool_bytes",
     "q4d_kv_pool_create", "q4d_kv_pool_destroy", "q4d_request_admit", "q4d_request_release", "q4d_request_len",
-    "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_profile_enable",
+    "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_decode_step_sampled", "q4d_sample", "q4d_profile_enable",
     "q4d_profile_read", "q4d_launch_count", "q4d_step_is_fused", "q4d_timeline_enable", "q4d_timeline_read",
     "q4d_step_io_bytes", "q4d_moe_touched_experts", "q4d_op_scratch_bytes", "q4d_q4_gemm",
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
@@ -235,6 +235,40 @@ def decode_step(model, pool, request_ids, last_tokens, block_tables, next_tokens
     toks = np.ascontiguousarray(last_tokens, dtype=np.int32)
     _check(lib().q4d_decode_step(model.handle, pool.handle, C.c_int32(ids.size), _ptr(ids), _ptr(toks), _ptr(bt),
                                  C.c_int32(bt.shape[1]), _ptr(next_tokens), _ptr(logits), _stream(stream)))
+
+
+class SamplingStruct(C.Structure):
+    _fields_ = [("temperature", C.c_void_p), ("top_k", C.c_void_p), ("top_p", C.c_void_p), ("u", C.c_void_p)]
+
+
+def _sampling(temperature, top_k, top_p, u):
+    """Host arrays of the per-request settings as a q4d_sampling (the arrays are returned too: keep them alive)."""
+    arrs = (np.ascontiguousarray(temperature, dtype=np.float32), np.ascontiguousarray(top_k, dtype=np.int32),
+            np.ascontiguousarray(top_p, dtype=np.float32), np.ascontiguousarray(u, dtype=np.float32))
+    st = SamplingStruct(*(a.ctypes.data for a in arrs))
+    return st, arrs
+
+
+def decode_step_sampled(model, pool, request_ids, last_tokens, block_tables, temperature, top_k, top_p, u,
+                        next_tokens, logits=None, stream=None):
+    """q4d_decode_step_sampled: the step, with next_tokens drawn by temperature / top-k / top-p from the given u."""
+    ids, bt = _step_args(request_ids, block_tables)
+    toks = np.ascontiguousarray(last_tokens, dtype=np.int32)
+    st, keep = _sampling(temperature, top_k, top_p, u)
+    _check(lib().q4d_decode_step_sampled(model.handle, pool.handle, C.c_int32(ids.size), _ptr(ids), _ptr(toks),
+                                         _ptr(bt), C.c_int32(bt.shape[1]), C.byref(st), _ptr(next_tokens),
+                                         _ptr(logits), _stream(stream)))
+    del keep
+
+
+def sample(logits, temperature, top_k, top_p, u, stream=None):
+    """q4d_sample on a device tensor of logits f32 [n][vocab]; returns the drawn tokens (device int32 [n])."""
+    out = torch.empty(logits.shape[0], dtype=torch.int32, device=logits.device)
+    st, keep = _sampling(temperature, top_k, top_p, u)
+    _check(lib().q4d_sample(_ptr(logits), C.c_int32(logits.shape[0]), C.c_int32(logits.shape[1]), C.byref(st),
+                            _ptr(out), _stream(stream)))
+    del keep
+    return out
 
 
 def decode_step_chained(model, pool, request_ids, last_tokens_device, block_tables, next_tokens, logits=None,

@@ -845,6 +845,49 @@ int q4d_decode_step(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* i
                    static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+int fill_sample_args(const q4d_sampling* sp, int n, int vocab, SampleArgs* a) {
+  if (!sp || !sp->temperature || !sp->top_k || !sp->top_p || !sp->u) return fail(Q4D_ERR_INVALID_ARG, "sampling: NULL argument");
+  for (int r = 0; r < n; ++r) {
+    if (!(sp->u[r] >= 0.0f && sp->u[r] < 1.0f)) return fail(Q4D_ERR_INVALID_ARG, "sampling: u[%d] outside [0, 1)", r);
+    if (sp->temperature[r] > 0.0f && !(sp->top_p[r] > 0.0f)) return fail(Q4D_ERR_INVALID_ARG, "sampling: top_p[%d] must be positive", r);
+    a->temperature[r] = sp->temperature[r], a->top_k[r] = sp->top_k[r], a->top_p[r] = sp->top_p[r], a->u[r] = sp->u[r];
+  }
+  for (int r = n; r < kMaxBatch; ++r) a->temperature[r] = 0.0f, a->top_k[r] = 0, a->top_p[r] = 1.0f, a->u[r] = 0.0f;
+  a->vocab = vocab;
+  return Q4D_OK;
+}
+}  // namespace
+
+int q4d_decode_step_sampled(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* last_tokens,
+                            const int32_t* bt, int32_t max_blocks, const q4d_sampling* sampling, int32_t* next_tokens,
+                            float* logits, void* stream) {
+  if (!m) return fail(Q4D_ERR_INVALID_ARG, "decode_step_sampled: NULL model");
+  if (n > 0 && !last_tokens) return fail(Q4D_ERR_INVALID_ARG, "decode_step_sampled: NULL last_tokens");
+  if (n < 0 || n > kMaxBatch) return fail(Q4D_ERR_BATCH_TOO_LARGE, "decode_step_sampled: n outside 0..16");
+  SampleArgs sa;
+  int rc = fill_sample_args(sampling, n, m->sh.vocab, &sa);
+  if (rc != Q4D_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  float* lg = logits ? logits : at<float>(m, m->lay.logits);  // the draw reads the logits: they are always produced
+  rc = step_impl(m, pool, n, ids, last_tokens, nullptr, bt, max_blocks, next_tokens, lg, s);
+  if (rc != Q4D_OK || n == 0) return rc;
+  sa.logits = lg, sa.next = next_tokens;
+  cudaError_t e = launch_sample(sa, n, s);
+  m->launches++;
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "sample");
+}
+
+int q4d_sample(const float* logits, int32_t n, int32_t vocab, const q4d_sampling* sampling, int32_t* next, void* stream) {
+  if (!logits || !next || n < 0 || n > kMaxBatch || vocab < 1) return fail(Q4D_ERR_INVALID_ARG, "sample: bad argument");
+  SampleArgs sa;
+  const int rc = fill_sample_args(sampling, n, vocab, &sa);
+  if (rc != Q4D_OK) return rc;
+  sa.logits = logits, sa.next = next;
+  cudaError_t e = launch_sample(sa, n, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "sample");
+}
+
 int q4d_decode_step_chained(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids,
                             const int32_t* last_tokens_device, const int32_t* bt, int32_t max_blocks,
                             int32_t* next_tokens, float* logits, void* stream) {

@@ -161,6 +161,18 @@ struct MoeCombineArgs {
 cudaError_t launch_moe_router(const MoeRouteArgs& a, int n, cudaStream_t s);
 cudaError_t launch_moe_combine(const MoeCombineArgs& a, int n, cudaStream_t s);
 
+// ---- sampling ------------------------------------------------------------------------
+struct SampleArgs {  // passed to the kernel by value: the per-request settings travel with the launch
+  const float* logits;  // f32 [n][vocab]
+  int32_t* next;        // [n]
+  int vocab;
+  float temperature[kMaxBatch];  // <= 0: greedy
+  int top_k[kMaxBatch];          // <= 0 or >= vocab: off
+  float top_p[kMaxBatch];        // >= 1: off
+  float u[kMaxBatch];            // the draw, in [0, 1)
+};
+cudaError_t launch_sample(const SampleArgs& a, int n, cudaStream_t s);
+
 // ---- small kernels ----------------------------------------------------------------
 cudaError_t launch_embed(const uint32_t* q, const uint16_t* scales, const uint16_t* biases, int vocab, int H,
                          const int32_t* tokens, int n, uint16_t* x, cudaStream_t s);
