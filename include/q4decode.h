@@ -211,6 +211,75 @@ int q4d_decode_step_host(q4d_model* model, q4d_kv_pool* pool, int32_t n, const i
                          const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
                          int32_t* next_tokens_host, float* logits_host, void* cuda_stream);
 
+/* ---- caches of the serving loop (host side) ------------------------------ */
+
+/* SHA-256 (FIPS 180-4) of a byte string, the hash both caches key on (Algorithm 2, Algorithm 3). */
+int q4d_sha256(const void* data, size_t bytes, uint8_t* out32);
+
+/* Text prefix cache (Algorithm 2, "Text Prefix Cache Lookup"; Section 3.2 "Text Prefix Caching").  The KV state of
+ * a prompt prefix is a list of 16-token blocks of the caller's pool; the cache stores one entry per block-aligned
+ * prefix, keyed by SHA-256(key of the prefix one block shorter || the block's 16 int32 token ids), so a lookup costs
+ * one hash per block and finds exactly the prefixes Algorithm 2 finds when it tries every prefix length from |P|
+ * down to 1: the longest cached one.  Entries are evicted least-recently-used first within a byte budget (Section
+ * 3.3, "Memory Management": 512 MB by default), never while a request reads them and never before the longer
+ * prefixes that build on them.  The cache owns no device memory: it deals in block ids.
+ *   capacity_bytes   0 = 512 MiB
+ *   bytes_per_block  what one block costs in the pool (all layers, K and V): q4d_kv_pool_bytes(shape, 1, 16) */
+typedef struct q4d_prefix_cache q4d_prefix_cache;
+int q4d_prefix_cache_create(size_t capacity_bytes, size_t bytes_per_block, q4d_prefix_cache** out);
+int q4d_prefix_cache_destroy(q4d_prefix_cache* cache);
+/* Longest cached prefix of the prompt (host tokens): its blocks (blocks_out) and one handle per block (handles_out),
+ * both [max_blocks]; *n_hit_blocks of them are filled, and generation resumes at position 16 * *n_hit_blocks
+ * (Algorithm 2's "start position"; 0 = miss).  The returned blocks are read-only for the caller and stay pinned
+ * until their handles are released. */
+int q4d_prefix_lookup(q4d_prefix_cache* cache, const int32_t* tokens, int32_t n_tokens, int32_t max_blocks,
+                      int32_t* blocks_out, int32_t* handles_out, int32_t* n_hit_blocks);
+/* After the prompt's KV is in the pool: offers the first n_blocks full blocks of the request's block table.  For
+ * block i, adopted_out[i] = 1 if the cache now (or already) holds exactly this block for this prefix (the caller
+ * must not free it while it is cached), 0 if the prefix was cached before with another block (the caller's block
+ * stays its own); handles_out[i] is a new pinned handle for blocks the call added, -1 otherwise. */
+int q4d_prefix_insert(q4d_prefix_cache* cache, const int32_t* tokens, int32_t n_tokens, const int32_t* block_table,
+                      int32_t n_blocks, int32_t* handles_out, int32_t* adopted_out);
+/* A request stops reading: its handles (negative ones are skipped) are unpinned. */
+int q4d_prefix_release(q4d_prefix_cache* cache, const int32_t* handles, int32_t n);
+/* Evicts least-recently-used unpinned leaf entries until the cache is within its budget and at least bytes_to_free
+ * bytes are gone (or nothing evictable is left, or max_out entries were evicted); the blocks given up are returned
+ * for the caller's allocator. */
+int q4d_prefix_evict(q4d_prefix_cache* cache, size_t bytes_to_free, int32_t max_out, int32_t* freed_blocks,
+                     int32_t* n_freed);
+int q4d_prefix_cache_stats(q4d_prefix_cache* cache, int64_t* entries, int64_t* bytes, int64_t* lookups,
+                           int64_t* hit_blocks);
+
+/* Content-hash store of the multimodal path (Algorithm 3, "Cache-Aware Multimodal Generation"; Section 3.3).  An
+ * image is identified by the SHA-256 of its decoded pixel bytes, whatever form it arrived in; an entry keeps what
+ * Algorithm 3 stores for reuse: the vision embeddings (a caller-owned device buffer) and the KV state (blocks of
+ * the pool).  The vision encoder itself is outside this library.  LRU eviction within a byte budget (0 = 512 MiB),
+ * never of an entry a request is using. */
+typedef struct {
+  uint8_t hash[32];   /* SHA-256 of the pixel bytes (filled by q4d_content_lookup) */
+  void* embeddings;   /* device buffer with the vision embeddings, owned by the caller */
+  int64_t bytes;      /* bytes the entry accounts for (embeddings + its KV blocks) */
+  int32_t n_tokens;   /* tokens of KV state stored with it */
+  int32_t n_blocks;   /* blocks of the pool holding that KV state */
+} q4d_content_entry;
+typedef struct q4d_content_cache q4d_content_cache;
+int q4d_content_cache_create(size_t capacity_bytes, q4d_content_cache** out);
+int q4d_content_cache_destroy(q4d_content_cache* cache);
+/* Hashes the pixels and looks the hash up.  *hit = 1: entry_out and blocks_out[0..n_blocks) hold the stored
+ * embeddings and KV state (skip the vision encoder and the prompt processing for this image) and the entry is
+ * pinned until q4d_content_release; *hit = 0: only entry_out->hash is filled, to be completed and stored. */
+int q4d_content_lookup(q4d_content_cache* cache, const void* pixels, size_t pixel_bytes, q4d_content_entry* entry_out,
+                       int32_t max_blocks, int32_t* blocks_out, int32_t* hit);
+/* Stores an entry after a miss (Algorithm 3, last step); it starts pinned by the storing request.
+ * DUPLICATE_REQUEST if the hash is present. */
+int q4d_content_store(q4d_content_cache* cache, const q4d_content_entry* entry, const int32_t* blocks);
+int q4d_content_release(q4d_content_cache* cache, const uint8_t* hash32);
+/* Evicts the least-recently-used unpinned entry if the store is over its budget or bytes_to_free > 0; *did_evict
+ * says whether one went, and evicted_out / blocks_out name what the caller may now free.  Call until *did_evict = 0. */
+int q4d_content_evict(q4d_content_cache* cache, size_t bytes_to_free, q4d_content_entry* evicted_out,
+                      int32_t max_blocks, int32_t* blocks_out, int32_t* did_evict);
+int q4d_content_cache_stats(q4d_content_cache* cache, int64_t* entries, int64_t* bytes);
+
 /* ---- instrumentation ---------------------------------------------------- */
 
 /* Kernel classes timed by the profile mode. */

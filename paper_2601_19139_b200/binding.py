@@ -26,6 +26,10 @@ EXPORTS = [
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
     "q4d_rmsnorm", "q4d_embed", "q4d_rope_append", "q4d_paged_attention", "q4d_argmax", "q4d_debug_dequant",
     "q4d_debug_kv_gather", "q4d_debug_run_layers", "q4d_debug_set_status",
+    "q4d_sha256", "q4d_prefix_cache_create", "q4d_prefix_cache_destroy", "q4d_prefix_lookup", "q4d_prefix_insert",
+    "q4d_prefix_release", "q4d_prefix_evict", "q4d_prefix_cache_stats", "q4d_content_cache_create",
+    "q4d_content_cache_destroy", "q4d_content_lookup", "q4d_content_store", "q4d_content_release", "q4d_content_evict",
+    "q4d_content_cache_stats",
 ]
 
 
@@ -401,3 +405,110 @@ def debug_run_layers(model, pool, request_ids, block_tables, layer_begin, layer_
                                       C.c_int32(bt.shape[1]), C.c_int32(layer_begin), C.c_int32(layer_end),
                                       _ptr(x_in), _ptr(x_out), _stream(stream)))
     return x_out
+
+
+# ---- caches of the serving loop (host side) ----------------------------------------------
+
+def sha256(data: bytes) -> bytes:
+    out = (C.c_uint8 * 32)()
+    _check(lib().q4d_sha256(data, C.c_size_t(len(data)), out))
+    return bytes(out)
+
+
+class PrefixCache:
+    """q4d_prefix_cache_*: the text prefix cache of Algorithm 2 over block ids."""
+
+    def __init__(self, capacity_bytes, bytes_per_block):
+        self.handle = C.c_void_p()
+        _check(lib().q4d_prefix_cache_create(C.c_size_t(capacity_bytes), C.c_size_t(bytes_per_block), C.byref(self.handle)))
+
+    def lookup(self, tokens):
+        """(blocks, handles) of the longest cached prefix; the start position is 16 * len(blocks)."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        mb = t.size // 16
+        blocks, handles, hit = np.zeros(max(mb, 1), dtype=np.int32), np.zeros(max(mb, 1), dtype=np.int32), C.c_int32()
+        _check(lib().q4d_prefix_lookup(self.handle, _ptr(t), C.c_int32(t.size), C.c_int32(mb), _ptr(blocks), _ptr(handles),
+                                       C.byref(hit)))
+        return blocks[:hit.value].tolist(), handles[:hit.value].tolist()
+
+    def insert(self, tokens, block_table):
+        """(handles, adopted) for the full blocks of the prompt."""
+        t = np.ascontiguousarray(tokens, dtype=np.int32)
+        bt = np.ascontiguousarray(block_table, dtype=np.int32)
+        nb = min(t.size // 16, bt.size)
+        handles, adopted = np.zeros(max(nb, 1), dtype=np.int32), np.zeros(max(nb, 1), dtype=np.int32)
+        _check(lib().q4d_prefix_insert(self.handle, _ptr(t), C.c_int32(t.size), _ptr(bt), C.c_int32(nb), _ptr(handles),
+                                       _ptr(adopted)))
+        return handles[:nb].tolist(), adopted[:nb].tolist()
+
+    def release(self, handles):
+        h = np.ascontiguousarray(handles, dtype=np.int32)
+        _check(lib().q4d_prefix_release(self.handle, _ptr(h), C.c_int32(h.size)))
+
+    def evict(self, bytes_to_free=0, max_out=1 << 16):
+        out, n = np.zeros(max_out, dtype=np.int32), C.c_int32()
+        _check(lib().q4d_prefix_evict(self.handle, C.c_size_t(bytes_to_free), C.c_int32(max_out), _ptr(out), C.byref(n)))
+        return out[:n.value].tolist()
+
+    def stats(self):
+        v = [C.c_int64() for _ in range(4)]
+        _check(lib().q4d_prefix_cache_stats(self.handle, *(C.byref(x) for x in v)))
+        return dict(zip(("entries", "bytes", "lookups", "hit_blocks"), (x.value for x in v)))
+
+    def close(self):
+        if self.handle:
+            lib().q4d_prefix_cache_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+
+class ContentEntry(C.Structure):
+    _fields_ = [("hash", C.c_uint8 * 32), ("embeddings", C.c_void_p), ("bytes", C.c_int64), ("n_tokens", C.c_int32),
+                ("n_blocks", C.c_int32)]
+
+
+class ContentCache:
+    """q4d_content_cache_*: the content-hash store of Algorithm 3 (embeddings handle + KV blocks per image hash)."""
+
+    def __init__(self, capacity_bytes, max_blocks=4096):
+        self.handle = C.c_void_p()
+        self.max_blocks = max_blocks
+        _check(lib().q4d_content_cache_create(C.c_size_t(capacity_bytes), C.byref(self.handle)))
+
+    def lookup(self, pixels: bytes):
+        """(hit, entry, blocks): on a miss the entry carries only the hash."""
+        e, hit = ContentEntry(), C.c_int32()
+        blocks = np.zeros(self.max_blocks, dtype=np.int32)
+        _check(lib().q4d_content_lookup(self.handle, pixels, C.c_size_t(len(pixels)), C.byref(e), C.c_int32(self.max_blocks),
+                                        _ptr(blocks), C.byref(hit)))
+        return bool(hit.value), e, blocks[:e.n_blocks].tolist() if hit.value else []
+
+    def store(self, entry, blocks):
+        b = np.ascontiguousarray(blocks, dtype=np.int32)
+        entry.n_blocks = b.size
+        _check(lib().q4d_content_store(self.handle, C.byref(entry), _ptr(b)))
+
+    def release(self, hash32: bytes):
+        _check(lib().q4d_content_release(self.handle, (C.c_uint8 * 32).from_buffer_copy(hash32)))
+
+    def evict(self, bytes_to_free=0):
+        """Evicted (entry, blocks) pairs, least recently used first, until the store is within its budget."""
+        gone = []
+        while True:
+            e, did = ContentEntry(), C.c_int32()
+            blocks = np.zeros(self.max_blocks, dtype=np.int32)
+            _check(lib().q4d_content_evict(self.handle, C.c_size_t(bytes_to_free), C.byref(e), C.c_int32(self.max_blocks),
+                                           _ptr(blocks), C.byref(did)))
+            if not did.value:
+                return gone
+            gone.append((e, blocks[:e.n_blocks].tolist()))
+            bytes_to_free = max(0, bytes_to_free - e.bytes)
+
+    def stats(self):
+        n, b = C.c_int64(), C.c_int64()
+        _check(lib().q4d_content_cache_stats(self.handle, C.byref(n), C.byref(b)))
+        return {"entries": n.value, "bytes": b.value}
+
+    def close(self):
+        if self.handle:
+            lib().q4d_content_cache_destroy(self.handle)
+            self.handle = C.c_void_p()

@@ -7,7 +7,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libq4decode.so")
-SOURCES = ["api.cu", "q4_gemm.cu", "q4_umma.cu", "attention.cu", "elementwise.cu", "moe.cu", "sampling.cu", "no_alloc.cu", "fused_step.cu"]
+SOURCES = ["api.cu", "q4_gemm.cu", "q4_umma.cu", "attention.cu", "elementwise.cu", "moe.cu", "sampling.cu", "no_alloc.cu", "fused_step.cu", "cache.cpp"]
 
 
 def _newest_source_mtime():
