@@ -172,6 +172,22 @@ int q4d_decode_step(q4d_model* model, q4d_kv_pool* pool, int32_t n, const int64_
                     const int32_t* last_tokens, const int32_t* block_tables, int32_t max_blocks,
                     int32_t* next_tokens, float* logits, void* cuda_stream);
 
+/* Prompt processing for one request (Section 3.2, "Text Prefix Caching": the forward pass over the prompt, which a
+ * cache hit skips for the cached tokens and resumes after them; Table 7 measures its latency as time to first
+ * token).  Computes K, V of tokens[start_pos .. n_tokens) at their positions, writes them into the request's blocks,
+ * and returns the greedy token that follows the prompt.  tokens and block_table are host arrays (block_table[i]
+ * holds tokens 16 i .. 16 i + 15 and must cover n_tokens; the blocks of positions < start_pos already hold their
+ * K, V, e.g. from q4d_prefix_lookup; a partly cached block that receives new tokens must be the request's own).
+ * next_token (device, 1 value) and logits (device f32 [vocab]) may be NULL.  The result is, by definition, what
+ * n_tokens - start_pos decode steps feeding the prompt's tokens one by one would leave behind; the library gets
+ * there sixteen tokens at a time (one pass over the weights per sixteen tokens, each token attending to the cached
+ * ones and to the earlier tokens of its chunk).  On success the request is admitted with n_tokens cached tokens.
+ * Errors: DUPLICATE_REQUEST (already admitted), POSITION_OVERFLOW, BLOCK_TABLE_TOO_SHORT, BLOCK_OUT_OF_RANGE,
+ * INVALID_ARG (start_pos outside [0, n_tokens): to reuse a fully cached prompt pass start_pos = n_tokens - 1). */
+int q4d_prefill(q4d_model* model, q4d_kv_pool* pool, int64_t request_id, const int32_t* tokens, int32_t n_tokens,
+                int32_t start_pos, const int32_t* block_table, int32_t max_blocks, int32_t* next_token, float* logits,
+                void* cuda_stream);
+
 /* Per-request sampling settings of one step (host arrays of n entries each, read before the call returns).  The
  * paper's scheduler only says that a token is generated per request (Algorithm 1, generation loop) and is silent on
  * how it is chosen; this is the usual temperature / top-k / top-p rule with the random draw supplied by the caller,

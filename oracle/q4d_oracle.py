@@ -282,6 +282,19 @@ class OracleModel:
         return nxt, logits, taps
 
 
+# ------------------------------------------------------------------ prompt processing
+def prefill(model, pool, block_size, tokens, start_pos, block_table):
+    """Prompt processing for one request (Section 3.2: the forward pass over the prompt tokens that a prefix-cache
+    hit skips up to start_pos).  By definition it is the decode step applied to the prompt's tokens one after the
+    other, each at its position, over the same pool: K, V of tokens[start_pos:] are appended in place, and the result
+    of the last step (greedy token after the prompt, its logits) is returned."""
+    bt = np.ascontiguousarray(block_table, dtype=np.int32).reshape(1, -1)
+    nxt = logits = None
+    for pos in range(int(start_pos), len(tokens)):
+        nxt, logits, _ = model.decode_step(pool, block_size, [pos], [int(tokens[pos])], bt)
+    return int(nxt[0]), logits[0]
+
+
 # ------------------------------------------------------------------ sampling
 # The paper's scheduler generates "a token" per request (Algorithm 1, generation loop) and says nothing about how
 # it is chosen.  The reading built here is the usual temperature / top-k / top-p rule with the random draw u given by

@@ -20,7 +20,7 @@ K_NAMES = ["embed", "rmsnorm", "gemm_qkv", "rope_append", "attention", "attn_mer
 EXPORTS = [
     "q4d_last_error", "q4d_model_workspace_bytes", "q4d_model_create", "q4d_model_destroy", "q4d_kv_pool_bytes",
     "q4d_kv_pool_create", "q4d_kv_pool_destroy", "q4d_request_admit", "q4d_request_release", "q4d_request_len",
-    "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_decode_step_sampled", "q4d_sample", "q4d_profile_enable",
+    "q4d_request_count", "q4d_decode_step", "q4d_decode_step_chained", "q4d_decode_step_host", "q4d_decode_step_sampled", "q4d_sample", "q4d_prefill", "q4d_profile_enable",
     "q4d_profile_read", "q4d_launch_count", "q4d_step_is_fused", "q4d_timeline_enable", "q4d_timeline_read",
     "q4d_step_io_bytes", "q4d_moe_touched_experts", "q4d_op_scratch_bytes", "q4d_q4_gemm",
     "q4d_q4_gemm_noalloc", "q4d_noalloc_max_scratch_bytes",
@@ -239,6 +239,15 @@ def decode_step(model, pool, request_ids, last_tokens, block_tables, next_tokens
     toks = np.ascontiguousarray(last_tokens, dtype=np.int32)
     _check(lib().q4d_decode_step(model.handle, pool.handle, C.c_int32(ids.size), _ptr(ids), _ptr(toks), _ptr(bt),
                                  C.c_int32(bt.shape[1]), _ptr(next_tokens), _ptr(logits), _stream(stream)))
+
+
+def prefill(model, pool, request_id, tokens, start_pos, block_table, next_token=None, logits=None, stream=None):
+    """q4d_prefill: processes tokens[start_pos:] of a prompt into the request's blocks and admits the request."""
+    t = np.ascontiguousarray(tokens, dtype=np.int32)
+    bt = np.ascontiguousarray(block_table, dtype=np.int32)
+    _check(lib().q4d_prefill(model.handle, pool.handle, C.c_int64(int(request_id)), _ptr(t), C.c_int32(t.size),
+                             C.c_int32(int(start_pos)), _ptr(bt), C.c_int32(bt.size), _ptr(next_token), _ptr(logits),
+                             _stream(stream)))
 
 
 class SamplingStruct(C.Structure):

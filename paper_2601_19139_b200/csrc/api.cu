@@ -441,15 +441,23 @@ struct LayerRange {
   uint16_t* x_out;
 };
 
+// Prompt processing: the n rows of the launch sequence are n consecutive tokens of ONE request, row r at position
+// start + r, all reading the same block table.  K, V of the rows are appended by a kernel of their own before the
+// attention kernel runs (a row attends to the rows before it), and only the last chunk of a prompt needs the head.
+struct PrefillRows {
+  int start;
+  bool want_head;
+};
+
 int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, const int32_t* tokens_host,
               const int32_t* tokens_dev, const int32_t* bt, int32_t max_blocks, int32_t* next_dev, float* logits_dev,
-              cudaStream_t s, const LayerRange* range = nullptr) {
+              cudaStream_t s, const LayerRange* range = nullptr, const PrefillRows* pf = nullptr) {
   if (!m || !pool || pool->model != m) return fail(Q4D_ERR_INVALID_ARG, "decode_step: model/pool mismatch or NULL");
   if (n < 0) return fail(Q4D_ERR_INVALID_ARG, "decode_step: n < 0");
   if (n == 0) return Q4D_OK;
   if (n > m->sh.max_batch)
     return fail(Q4D_ERR_BATCH_TOO_LARGE, "decode_step: n = %d exceeds max_batch %d", n, m->sh.max_batch);
-  if (!ids || !bt || max_blocks < 1 || (!range && ((!tokens_host && !tokens_dev) || !next_dev)))
+  if ((!ids && !pf) || !bt || max_blocks < 1 || (!range && ((!tokens_host && !tokens_dev) || !next_dev)))
     return fail(Q4D_ERR_INVALID_ARG, "decode_step: NULL argument");
   const q4d_shape& sh = m->sh;
   {
@@ -459,7 +467,9 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
 
   // ---- validate on the host; nothing is changed before this block passes ----
   int32_t lens[kMaxBatch];
-  {
+  if (pf) {  // validated by the caller (q4d_prefill): one request, consecutive positions
+    for (int r = 0; r < n; ++r) lens[r] = pf->start + r;
+  } else {
     std::unordered_set<int64_t> seen;
     for (int r = 0; r < n; ++r) {
       const long long id = (long long)ids[r];
@@ -504,11 +514,11 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     h_tokens[r] = tokens_host ? tokens_host[r] : 0;
     h_lens[r] = lens[r];
     const int need = (lens[r] + 1 + kBlockSize - 1) / kBlockSize;  // <= max_blocks_cap since len < max_positions
-    for (int i = 0; i < ml.max_blocks_cap; ++i)
-      h_bt[(size_t)r * ml.max_blocks_cap + i] = i < need ? bt[(size_t)r * max_blocks + i] : 0;
+    const int32_t* bt_row = bt + (pf ? 0 : (size_t)r * max_blocks);
+    for (int i = 0; i < ml.max_blocks_cap; ++i) h_bt[(size_t)r * ml.max_blocks_cap + i] = i < need ? bt_row[i] : 0;
   }
   AttnPlan plan = {0, 0, 0};  // the whole-step kernel plans its attention items from the lengths alone
-  if (!m->fused) plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
+  if (!m->fused || pf) plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
   unsigned char* dmeta = m->ws + m->lay.meta;
   const size_t head_bytes = ml.off_work + (size_t)plan.n_work * sizeof(int4);
   const size_t bt_bytes = (size_t)n * ml.max_blocks_cap * 4;
@@ -524,7 +534,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   const int32_t* d_lens = reinterpret_cast<const int32_t*>(dmeta + ml.off_lens);
   const int32_t* d_bt = reinterpret_cast<const int32_t*>(dmeta + ml.off_bt);
 
-  if (m->fused) {
+  if (m->fused && !pf) {
     const int rc = run_fused(m, pool, n, lens, d_tokens, d_bt, next_dev, logits_dev, s, range ? range->begin : 0,
                              range ? range->end : 0, range ? range->x_in : nullptr, range ? range->x_out : nullptr,
                              range != nullptr);
@@ -585,6 +595,15 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     // q preparation (qk-norm, rotary embedding) and the append of k, v happen inside the attention kernel
     aa.qkv = qkv, aa.q_norm = sh.qk_norm ? lw.q_norm : nullptr, aa.k_norm = sh.qk_norm ? lw.k_norm : nullptr;
     aa.eps = sh.rms_eps, aa.rope = m->w.rope_cos_sin, aa.kpool_w = kpool, aa.vpool_w = vpool;
+    if (pf) {
+      // prompt rows: append k, v of all rows first; the attention kernel then starts after that kernel has ended
+      RopeArgs ra;
+      ra.qkv = qkv, ra.q_norm = aa.q_norm, ra.k_norm = aa.k_norm, ra.eps = sh.rms_eps, ra.rope = m->w.rope_cos_sin;
+      ra.n = n, ra.nq = nq, ra.nkv = nkv, ra.lens = d_lens, ra.block_tables = d_bt, ra.max_blocks = ml.max_blocks_cap;
+      ra.kpool = kpool, ra.vpool = vpool, ra.q_out = qbuf;
+      Q4D_LAUNCH(Q4D_K_ROPE_APPEND, launch_rope_append(ra, s));
+      aa.qkv = nullptr, aa.after_predecessor = true;
+    }
     Q4D_LAUNCH(Q4D_K_ATTENTION, launch_paged_attention(aa, s));
     Q4D_LAUNCH(Q4D_K_GEMM_O, launch_q4_gemm(gemm_args(m, lw.wo, H, qdim, ap, as, n, EPI_RESIDUAL, x, H), s));
     if (sh.n_experts == 0) {
@@ -627,6 +646,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     cudaError_t ce = cudaMemcpyAsync(range->x_out, x, (size_t)n * H * 2, cudaMemcpyDeviceToDevice, s);
     return ce == cudaSuccess ? Q4D_OK : fail_cuda(ce, "hidden state copy");
   }
+  if (pf && !pf->want_head) return Q4D_OK;  // an inner chunk of a prompt: its K, V are in the pool, nothing else is needed
   Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, m->w.final_norm, sh.rms_eps, n, H, nullptr, yp, ys, dense_layout, s));
   GemmArgs lm = gemm_args(m, m->w.lm_head, V, H, yp, ys, n, EPI_F32, logits, V);
   lm.argmax_partial = amax;
@@ -642,7 +662,8 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     m->status_pending = true;
   }
 
-  for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
+  if (!pf)
+    for (int r = 0; r < n; ++r) pool->lens[ids[r]] = lens[r] + 1;
   return Q4D_OK;
 }
 
@@ -886,6 +907,48 @@ int q4d_sample(const float* logits, int32_t n, int32_t vocab, const q4d_sampling
   sa.logits = logits, sa.next = next;
   cudaError_t e = launch_sample(sa, n, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? Q4D_OK : fail_cuda(e, "sample");
+}
+
+int q4d_prefill(q4d_model* m, q4d_kv_pool* pool, int64_t request_id, const int32_t* tokens, int32_t n_tokens,
+                int32_t start_pos, const int32_t* block_table, int32_t max_blocks, int32_t* next_token, float* logits,
+                void* stream) {
+  if (!m || !pool || pool->model != m) return fail(Q4D_ERR_INVALID_ARG, "prefill: model/pool mismatch or NULL");
+  if (!tokens || !block_table || n_tokens < 1 || start_pos < 0 || start_pos >= n_tokens || max_blocks < 1)
+    return fail(Q4D_ERR_INVALID_ARG, "prefill: need 0 <= start_pos < n_tokens and a block table");
+  const q4d_shape& sh = m->sh;
+  if (n_tokens >= sh.max_positions)
+    return fail(Q4D_ERR_POSITION_OVERFLOW, "prefill: %d tokens do not leave a position to generate at (max_positions %d)",
+                n_tokens, sh.max_positions);
+  if (pool->lens.count(request_id))
+    return fail(Q4D_ERR_DUPLICATE_REQUEST, "prefill: request %lld already admitted", (long long)request_id);
+  const int need = (n_tokens + kBlockSize - 1) / kBlockSize;
+  if (need > max_blocks)
+    return fail(Q4D_ERR_BLOCK_TABLE_TOO_SHORT, "prefill: %d tokens need %d blocks, table has %d", n_tokens, need, max_blocks);
+  for (int i = 0; i < need; ++i)
+    if (block_table[i] < 0 || block_table[i] >= pool->num_blocks)
+      return fail(Q4D_ERR_BLOCK_OUT_OF_RANGE, "prefill: block %d = %d outside the pool", i, block_table[i]);
+  for (int t = start_pos; t < n_tokens; ++t)
+    if (tokens[t] < 0 || tokens[t] >= sh.vocab) return fail(Q4D_ERR_INVALID_ARG, "prefill: token %d outside the vocabulary", tokens[t]);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* ws_next = at<int32_t>(m, m->lay.next);
+  float* ws_logits = at<float>(m, m->lay.logits);
+  int last_rows = 0;
+  for (int c = start_pos; c < n_tokens; c += kMaxBatch) {
+    const int n = std::min(kMaxBatch, n_tokens - c);
+    const PrefillRows pf{c, c + n == n_tokens};
+    const int rc = step_impl(m, pool, n, nullptr, tokens + c, nullptr, block_table, max_blocks, ws_next,
+                             pf.want_head ? ws_logits : nullptr, s, nullptr, &pf);
+    if (rc != Q4D_OK) return rc;
+    last_rows = n;
+  }
+  cudaError_t e = cudaSuccess;
+  if (next_token) e = cudaMemcpyAsync(next_token, ws_next + (last_rows - 1), sizeof(int32_t), cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess && logits)
+    e = cudaMemcpyAsync(logits, ws_logits + (size_t)(last_rows - 1) * sh.vocab, (size_t)sh.vocab * sizeof(float),
+                        cudaMemcpyDeviceToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(e, "prefill outputs");
+  pool->lens[request_id] = n_tokens;
+  return Q4D_OK;
 }
 
 int q4d_decode_step_chained(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids,

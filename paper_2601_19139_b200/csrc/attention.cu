@@ -499,7 +499,7 @@ cudaError_t launch_paged_attention(const AttnArgs& a, cudaStream_t s) {
   const int G = a.nq / a.nkv;
   if (G < 1 || G > 16 || a.nq % a.nkv) return cudaErrorInvalidValue;
   const dim3 grid(a.n_work, a.nkv), block(kAttnThreads);
-  return launch_kernel(paged_attention_kernel, grid, block, kAttnWarps * kAttnStages * kAttnStage, s, a);
+  return launch_kernel_pdl(!a.after_predecessor, paged_attention_kernel, grid, block, kAttnWarps * kAttnStages * kAttnStage, s, a);
 }
 
 cudaError_t launch_attention_merge(const AttnArgs& a, cudaStream_t s) {

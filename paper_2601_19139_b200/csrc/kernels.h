@@ -106,6 +106,10 @@ struct AttnArgs {
   float* out_xs;    // its group sums [nq*2][16]
   int out_layout = OPERAND_ROWS;  // layout of out_xp
   int* merge_counters = nullptr;  // [16][nkv], zero between launches: the attention kernel merges the chunks itself
+  // The kernel requests its first K, V tiles before it waits for the preceding kernel (cached K, V do not depend on
+  // it).  Set when they do (the preceding kernel appends tokens this launch reads): the launch then carries no
+  // programmatic-dependent-launch attribute and starts only after the preceding kernel has completed.
+  bool after_predecessor = false;
   // With qkv given (bf16 [n][(nq+2nkv)*128], the QKV projection's output) the kernel prepares q itself (qk-norm,
   // rotary embedding) and appends k, v of the new token to the pool; `q` is then unused.
   const uint16_t* qkv = nullptr;
