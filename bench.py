@@ -314,6 +314,44 @@ def main():
     ms_e2e_lg = (time.perf_counter() - t_host0) * 1e3
     h2d_lg, d2h_lg = model.step_io_bytes()
 
+    # ---- the neighbouring rows of the path, on the same model: prompt processing and sampling ----
+    def timed_ms(fn, reps=3):
+        best = 1e30
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        return best
+
+    extras = {}
+    try:
+        prompt = np.random.default_rng(seed + 5).integers(0, shape.vocab, size=512).astype(np.int32)
+        pblocks = script.alloc.alloc(33)
+        rid = [10 ** 9]
+
+        def run_prefill(start):
+            q4d.prefill(model, pool, rid[0], prompt, start, pblocks)
+            pool.request_release(rid[0])
+            rid[0] += 1
+
+        t_full = timed_ms(lambda: run_prefill(0))
+        t_hit = timed_ms(lambda: run_prefill(496))       # a 496-token prefix already cached: 16 tokens to process
+        extras["prefill"] = {"prompt_tokens": 512, "ttft_ms": t_full, "tokens_per_s": 512 / (t_full * 1e-3),
+                             "ttft_ms_with_496_cached": t_hit, "speedup_from_prefix_cache": t_full / t_hit,
+                             "note": "q4d_prefill: sixteen tokens per pass over the weights (not a compute-bound "
+                                     "kernel yet); the paper's Table 7 reports 245 ms -> 42 ms on its hardware"}
+        script.alloc.release(pblocks)
+        lg = torch.randn(n, shape.vocab, device=device)
+        us = np.random.default_rng(seed + 6).uniform(0, 1, size=n).astype(np.float32)
+        t_s = timed_ms(lambda: q4d.sample(lg, [0.8] * n, [50] * n, [0.95] * n, us), reps=5)
+        extras["sampling"] = {"us_per_step": t_s * 1e3, "settings": "temperature 0.8, top-k 50, top-p 0.95",
+                              "share_of_step": t_s / (ms / args.steps)}
+    except Exception as ex:  # the headline numbers do not depend on these
+        extras["error"] = repr(ex)
+
     # ---- per-launch timing (events around every launch) for the roofline of the dominant kernel ----
     fused = model.is_fused()
     model.profile_enable(True)
@@ -438,6 +476,7 @@ def main():
                             "returns": "next tokens and the fp32 logits of every request"},
         "gpu_launches": launches,
         "clocks": clocks,
+        "extras": extras,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
