@@ -142,6 +142,40 @@ def aggregate_ranks(dist, device, ms, ms_e2e, tokens, tokens_e2e, launches):
     return float(t[0]), float(t[1]), int(c[0]), int(c[1]), int(c[2])
 
 
+def gemm_only(args):
+    """One projection shape alone, for kernel-level timing and ncu captures: `--steps` calls of q4d_q4_gemm (operand
+    rearrangement + the projection kernel), CUDA events around the loop, one JSON line."""
+    import torch
+
+    from paper_2601_19139_b200 import binding as q4d
+    from paper_2601_19139_b200 import build as cuda_build
+    from workload import gen
+    cuda_build.build()
+    N, K = (int(v) for v in args.gemm.lower().split("x"))
+    n = args.gemm_batch
+    torch.cuda.set_device(0)
+    ws = [gen.random_q4(N, K, "cuda", "bench-gemm", N, K, i) for i in range(args.gemm_buffers)]
+    x = torch.randn((n, K), generator=torch.Generator(device="cpu").manual_seed(args.seed)).to(torch.bfloat16).cuda()
+    out = torch.empty(n, N, dtype=torch.float32, device="cuda")
+    for i in range(max(args.warmup, 3)):
+        q4d.q4_gemm(ws[i % len(ws)], x, n, epilogue=2, out=out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        q4d.q4_gemm(ws[i % len(ws)], x, n, epilogue=2, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / args.steps
+    by = N * K * 0.5625
+    peak, kind = peaks()
+    print(json.dumps({"op": "q4_gemm", "N": N, "K": K, "n": n, "epilogue": "f32", "calls": args.steps,
+                      "kernel": "q4_umma_kernel" if os.environ.get("Q4D_GEMM_KERNEL") == "tcgen05" else "span/round",
+                      "us_per_call": us, "GBps": by / us / 1e3, "frac_of_peak": by / us / 1e3 / peak, "peak_kind": kind,
+                      "note": "a call = operand rearrangement kernel + projection kernel"}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -153,7 +187,13 @@ def main():
     ap.add_argument("--oracle-budget", type=float, default=20.0, help="seconds of oracle steps in the CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--gemm", default=None, metavar="NxK",
+                    help="time one 4-bit projection of this shape alone (q4d_q4_gemm, fp32 outputs) instead of the step")
+    ap.add_argument("--gemm-batch", type=int, default=16)
+    ap.add_argument("--gemm-buffers", type=int, default=1, help="rotate over this many weight tensors (defeats L2)")
     args = ap.parse_args()
+    if args.gemm:
+        return gemm_only(args)
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

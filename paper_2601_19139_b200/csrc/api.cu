@@ -144,7 +144,8 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
     w.yplain = take(B * s.hidden * 2);
     w.m_idx = take(B * s.top_k * 4);
     w.m_wgt = take(B * s.top_k * 4);
-    w.m_ints = take((3 * E + 3) * 4);  // flags[E], expert_ids[E], slot_of[E], counter, n_touched, touched_total
+    // flags[E], expert_ids[E], slot_of[E], counter, n_touched, touched_total, slice_counter[16], then logits[16][E]
+    w.m_ints = take((3 * E + 3 + kMaxBatch) * 4 + B * E * 4);
     w.m_hp = take(E * B * s.expert_inter * 2);
     w.m_hs = take(E * (size_t)(s.expert_inter / 64) * 16 * 4);
     w.m_o = take(E * B * s.hidden * 2);
@@ -622,6 +623,8 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       mr.flags = ints, mr.expert_ids = ints + E, mr.slot_of = ints + 2 * E, mr.counter = ints + 3 * E;
       mr.n_touched = ints + 3 * E + 1;
       mr.touched_total = ints + 3 * E + 2;
+      mr.slice_counter = ints + 3 * E + 3;
+      mr.logits = reinterpret_cast<float*>(ints + 3 * E + 3 + kMaxBatch);
       uint16_t* ehp = at<uint16_t>(m, m->lay.m_hp);
       float* ehs = at<float>(m, m->lay.m_hs);
       uint16_t* eo = at<uint16_t>(m, m->lay.m_o);
@@ -748,7 +751,7 @@ int q4d_model_create(const q4d_shape* shape, const q4d_weights* weights, void* w
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.counters, 0, (size_t)lay.counters_len * 4);
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.attn_merge_counters, 0, (size_t)16 * shape->n_kv_heads * 4);
   if (e == cudaSuccess && shape->n_experts)
-    e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 3) * 4);
+    e = cudaMemset(m->ws + lay.m_ints, 0, (3 * (size_t)shape->n_experts + 3 + kMaxBatch) * 4);
   if (e == cudaSuccess) e = cudaMemset(m->ws + lay.chain_status, 0, 256);
   if (e == cudaSuccess) e = cudaMallocHost(reinterpret_cast<void**>(&m->host_status), sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&m->status_done, cudaEventDisableTiming);

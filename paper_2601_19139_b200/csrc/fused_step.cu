@@ -84,7 +84,6 @@ __device__ __forceinline__ int atom_acq_rel_add_s32(int* p, int v) {
   asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
   return old;
 }
-__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 
 // ---- mbarrier + 1-D bulk copy (global -> shared), used to stage the activations
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {

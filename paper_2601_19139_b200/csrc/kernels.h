@@ -152,6 +152,8 @@ struct MoeRouteArgs {
   int32_t* expert_ids;  // [E] touched experts, ascending
   int32_t* slot_of;     // [E] position of an expert in expert_ids
   int32_t* n_touched;
+  float* logits;           // [16][E] scratch
+  int32_t* slice_counter;  // [16], zero between launches
   int32_t* touched_total = nullptr;  // optional: running sum of n_touched over the launches of a step
 };
 struct MoeCombineArgs {

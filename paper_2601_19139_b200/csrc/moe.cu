@@ -20,32 +20,70 @@ namespace {
 
 constexpr int kMaxExperts = 256;
 
-// One CTA per request.  The last CTA to finish compacts the touched-expert flags into a list.
-__global__ void __launch_bounds__(256) moe_router_kernel(const MoeRouteArgs p) {
+constexpr int kRouterThreads = 256;
+constexpr int kRouterWarps = kRouterThreads / 32;
+
+// CTA (slice, request): the request's row is staged in shared memory and each warp computes the logits of one or
+// more experts of the slice, keeping eight 16-byte loads of a router row in flight per lane (the router matrix is
+// small, 512 KB for 128 experts of width 2048, so it is spread over many SMs and the loads overlap).  A lane adds
+// its chunks lane, lane + 32, ... in ascending order.  The logits go to global memory; the CTA that finishes a
+// request's last slice selects its experts, and the CTA that finishes the last request compacts the touched-expert
+// flags into a list.
+__global__ void __launch_bounds__(kRouterThreads) moe_router_kernel(const MoeRouteArgs p) {
+  extern __shared__ __align__(16) unsigned char router_smem[];
+  uint4* sy = reinterpret_cast<uint4*>(router_smem);  // the row: H / 8 chunks of 8 bf16
   __shared__ float sz[kMaxExperts];
   __shared__ int s_last;
-  __shared__ int s_warp_base[8];
+  __shared__ int s_warp_base[kRouterWarps];
   grid_launch_dependents();
-  grid_dependency_wait();
-  const int r = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint16_t* y = p.y + (size_t)r * p.H;
+  const int r = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunks = p.H >> 3;
-  for (int e = warp; e < p.E; e += 8) {
-    const uint16_t* wr = p.router + (size_t)e * p.H;
+  const int per_slice = (p.E + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int e_begin = blockIdx.x * per_slice, e_end = min(p.E, e_begin + per_slice);
+  grid_dependency_wait();
+  {
+    const uint4* y = reinterpret_cast<const uint4*>(p.y + (size_t)r * p.H);
+    for (int c = threadIdx.x; c < chunks; c += kRouterThreads) sy[c] = y[c];
+  }
+  __syncthreads();
+  for (int e = e_begin + warp; e < e_end; e += kRouterWarps) {
+    const uint4* wr = reinterpret_cast<const uint4*>(p.router + (size_t)e * p.H);
     float acc = 0.0f;
-    for (int c = lane; c < chunks; c += 32) {
-      const uint4 a = *reinterpret_cast<const uint4*>(wr + c * 8);
-      const uint4 b = *reinterpret_cast<const uint4*>(y + c * 8);
-      const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+    for (int c0 = lane; c0 < chunks; c0 += 32 * 8) {
+      uint4 a[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        acc = fmaf(bf16_lo(aw[i]), bf16_lo(bw[i]), acc);
-        acc = fmaf(bf16_hi(aw[i]), bf16_hi(bw[i]), acc);
+      for (int i = 0; i < 8; ++i) {
+        const int c = c0 + 32 * i;
+        a[i] = c < chunks ? __ldg(wr + c) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = c0 + 32 * i;
+        if (c < chunks) {
+          const uint4 b = sy[c];
+          const uint32_t aw[4] = {a[i].x, a[i].y, a[i].z, a[i].w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            acc = fmaf(bf16_lo(aw[j]), bf16_lo(bw[j]), acc);
+            acc = fmaf(bf16_hi(aw[j]), bf16_hi(bw[j]), acc);
+          }
+        }
       }
     }
     acc = warp_sum(acc);
-    if (lane == 0) sz[e] = acc;
+    if (lane == 0) p.logits[(size_t)r * p.E + e] = acc;
   }
+  // ---- the CTA with the request's last slice selects the experts ----
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    s_last = (atomicAdd(p.slice_counter + r, 1) == (int)gridDim.x - 1);
+    if (s_last) p.slice_counter[r] = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int e = threadIdx.x; e < p.E; e += kRouterThreads) sz[e] = __ldcg(p.logits + (size_t)r * p.E + e);
   __syncthreads();
   if (warp == 0) {
     // each lane owns experts lane, lane + 32, ...
@@ -98,7 +136,7 @@ __global__ void __launch_bounds__(256) moe_router_kernel(const MoeRouteArgs p) {
   // ---- the last CTA builds the list of touched experts, in ascending expert order ----
   __threadfence();
   __syncthreads();
-  if (threadIdx.x == 0) s_last = (atomicAdd(p.counter, 1) == (int)gridDim.x - 1);
+  if (threadIdx.x == 0) s_last = (atomicAdd(p.counter, 1) == (int)gridDim.y - 1);
   __syncthreads();
   if (!s_last) return;
   __threadfence();
@@ -117,7 +155,7 @@ __global__ void __launch_bounds__(256) moe_router_kernel(const MoeRouteArgs p) {
   if (e < p.E) p.flags[e] = 0;
   if (threadIdx.x == 0) {
     int tot = 0;
-    for (int w = 0; w < 8; ++w) tot += s_warp_base[w];
+    for (int w = 0; w < kMaxExperts / 32; ++w) tot += s_warp_base[w];
     *p.n_touched = tot;
     *p.counter = 0;
     if (p.touched_total) *p.touched_total += tot;  // one CTA per launch, launches of a step are stream-ordered
@@ -160,7 +198,9 @@ __global__ void __launch_bounds__(256) moe_combine_kernel(const MoeCombineArgs p
 cudaError_t launch_moe_router(const MoeRouteArgs& a, int n, cudaStream_t s) {
   if (n <= 0) return cudaSuccess;
   if (a.E < 1 || a.E > kMaxExperts || a.top_k < 1 || a.top_k > 32 || a.top_k > a.E || a.H % 8) return cudaErrorInvalidValue;
-  return launch_kernel(moe_router_kernel, dim3(n), dim3(256), 0, s, a);
+  if ((size_t)a.H * 2 > 48 * 1024 || !a.logits || !a.slice_counter) return cudaErrorInvalidValue;
+  const int slices = (a.E + kRouterWarps - 1) / kRouterWarps;  // one expert per warp while that gives at most 32 slices
+  return launch_kernel(moe_router_kernel, dim3(slices < 32 ? slices : 32, n), dim3(kRouterThreads), (size_t)a.H * 2, s, a);
 }
 
 cudaError_t launch_moe_combine(const MoeCombineArgs& a, int n, cudaStream_t s) {
