@@ -326,6 +326,7 @@ def main():
     for _ in range(args.steps):
         tokens += one_step("chained")
     e1.record(stream)
+    host_enqueue_ms = (time.time() - wall0) * 1e3 / args.steps   # host time to submit a step (the device lags behind)
     barrier()
     wall1 = time.time()
     ms = e0.elapsed_time(e1)
@@ -516,6 +517,7 @@ def main():
                             "returns": "next tokens and the fp32 logits of every request"},
         "gpu_launches": launches,
         "clocks": clocks,
+        "host_enqueue_ms_per_step": host_enqueue_ms,
         "extras": extras,
     }
 

@@ -519,7 +519,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
     for (int i = 0; i < ml.max_blocks_cap; ++i) h_bt[(size_t)r * ml.max_blocks_cap + i] = i < need ? bt_row[i] : 0;
   }
   AttnPlan plan = {0, 0, 0};  // the whole-step kernel plans its attention items from the lengths alone
-  if (!m->fused || pf) plan = plan_attention(lens, n, sh.n_kv_heads, 0, m->sm_count, h_work, h_slot, h_nch, ml.max_work);
+  if (!m->fused || pf) plan = plan_attention(lens, n, sh.n_kv_heads, 0, attention_wave_ctas(sh.n_q_heads, sh.n_kv_heads), h_work, h_slot, h_nch, ml.max_work);
   unsigned char* dmeta = m->ws + m->lay.meta;
   const size_t head_bytes = ml.off_work + (size_t)plan.n_work * sizeof(int4);
   const size_t bt_bytes = (size_t)n * ml.max_blocks_cap * 4;
@@ -1135,16 +1135,13 @@ int q4d_paged_attention(const uint16_t* q, const uint16_t* kpool, const uint16_t
     return fail(Q4D_ERR_INVALID_ARG, "paged_attention: bad head counts or batch");
   if (n == 0) return Q4D_OK;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  int sms = 148, dev = 0;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const size_t by_meta = (kOpAttnMeta - 1024) / sizeof(int4);
   const size_t by_acc = kOpPartAcc / ((size_t)nq * kHeadDim * 4), by_ml = kOpPartMl / ((size_t)nq * 8);
   const int max_work = (int)std::min(by_meta, std::min(by_acc, by_ml));
   std::vector<int4> work(max_work);
   int32_t head[2 * kMaxBatch];
   const AttnPlan plan =
-      plan_attention(lens_host, n, nkv, chunk_tokens, sms, work.data(), head, head + kMaxBatch, max_work);
+      plan_attention(lens_host, n, nkv, chunk_tokens, attention_wave_ctas(nq, nkv), work.data(), head, head + kMaxBatch, max_work);
   long long want = 0;
   for (int r = 0; r < n; ++r) want += ((lens_host[r] + 1 + 15) / 16 + plan.chunk_tiles - 1) / plan.chunk_tiles;
   if (want != plan.n_work)

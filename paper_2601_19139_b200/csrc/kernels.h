@@ -85,8 +85,10 @@ struct AttnPlan {   // filled on the host from the request lengths
   int chunk_tiles;  // tiles (16 tokens) per chunk
 };
 // work: int4 {request, first tile, end tile, slot}; slot_base/nchunks per request.
-AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, int sm_count, int4* work,
+// wave_ctas: CTAs resident at once (attention_wave_ctas); the automatic chunk size fills one such wave.
+AttnPlan plan_attention(const int32_t* lens, int n, int nkv, int chunk_tokens, int wave_ctas, int4* work,
                         int32_t* slot_base, int32_t* nchunks, int max_work);
+int attention_wave_ctas(int nq, int nkv);
 int attention_max_work(int max_batch, int max_positions);
 
 struct AttnArgs {

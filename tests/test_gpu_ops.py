@@ -265,6 +265,10 @@ def test_rope_append_matches_oracle(q4d, nq, nkv, qk_norm):
     # more than eight chunks per request: eleven 12-tile chunks with a 3-tile tail, and nine planner-sized chunks
     (32, 4, [1953, 194, 1036], 192),
     (32, 8, [9000, 40], 0),
+    # a full batch on four kv heads: the planner's one-wave chunking gives a request dozens of chunks across the
+    # three resident CTAs per SM; and a group of five query heads (columns 5..7 of the token-major MMA stay empty)
+    (32, 4, [8191, 5003, 3100, 2047, 1500, 1024, 1023, 777, 512, 300, 255, 129, 64, 17, 1, 0], 0),
+    (40, 8, [1200, 31, 640], 0),
 ])
 def test_paged_attention_matches_oracle(q4d, nq, nkv, lens, chunk):
     n = len(lens)

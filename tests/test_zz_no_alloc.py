@@ -7,6 +7,8 @@ so the test calls it twice in a row with different shapes and checks each result
 entry point q4d_q4_gemm, which runs the same kernel on caller-provided scratch: the results must be
 identical.  This file sorts last so that a run stopping at the first failure has run everything else.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -44,13 +46,19 @@ def test_noalloc_gemm_equals_the_scratch_taking_entry_point_twice_in_a_row(q4d):
     # driver); the calls under test come after it
     q4d.q4_gemm_noalloc(prepared[1][0], prepared[1][1], prepared[1][2], prepared[1][4], epilogue=prepared[1][3])
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
-    free_before = torch.cuda.mem_get_info()[0]
-    for w, x, n, epi, out in prepared:                     # two calls in a row on the shared array
-        q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
-    torch.cuda.synchronize()
-    assert torch.cuda.memory_allocated() == before
-    assert torch.cuda.mem_get_info()[0] == free_before     # nor did anything else take device memory
+    # tensors of earlier tests that only the cycle collector can free must not be freed between the two readings
+    gc.collect()
+    gc.disable()
+    try:
+        before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]
+        for w, x, n, epi, out in prepared:                 # two calls in a row on the shared array
+            q4d.q4_gemm_noalloc(w, x, n, out, epilogue=epi)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == before
+        assert torch.cuda.mem_get_info()[0] == free_before  # nor did anything else take device memory
+    finally:
+        gc.enable()
     for w, x, n, epi, out in prepared:
         want = q4d.q4_gemm(w, x, n, epilogue=epi)
         torch.cuda.synchronize()
