@@ -597,12 +597,15 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   grid_dependency_wait();
 
   // One bulk copy per request row of the slice (and one for its group sums), tracked by the buffer's mbarrier.
-  const uint32_t slice_bytes = (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0));
+  // Only the rows of requests that exist are fetched; the other columns of the MMAs multiply whatever the buffer
+  // holds and their results are never stored.
+  const int rows_used = p.n < NP ? p.n : NP;
+  const uint32_t slice_bytes = (uint32_t)(rows_used * ks * 2 + (p.xs ? sum_bytes : 0));
   auto stage_acts = [&](int gstep) {  // the lanes of warp 0 issue the copies side by side
     if (warp == 0) {
       const int buf = gstep & 1, slice = blockIdx.y * S + gstep % S;
       if (lane == 0) mbar_expect_tx(&s_mbar[buf], slice_bytes);
-      if (lane < NP)
+      if (lane < rows_used)
         bulk_copy_g2s(sAct + buf * act_bytes + lane * b_stride, p.xp + (size_t)lane * p.K + (size_t)slice * ks,
                       (uint32_t)(ks * 2), &s_mbar[buf]);
       else if (lane == NP && p.xs)
@@ -953,14 +956,17 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
   // every slice of the operand (and its group sums): one bulk copy per request row, all on one mbarrier, issued by
   // the lanes of warp 0 side by side (a single thread would spend microseconds issuing up to 68 copies)
   if (warp == 0) {
-    if (lane == 0) mbar_expect_tx(&s_mbar, (uint32_t)(NP * ks * 2 + (p.xs ? sum_bytes : 0)) * (uint32_t)S);
+    // only the rows of requests that exist are fetched: the other columns of the MMAs multiply whatever the buffer
+    // holds and their results are never stored
+    const int rows_used = p.n < NP ? p.n : NP;
+    if (lane == 0) mbar_expect_tx(&s_mbar, (uint32_t)(rows_used * ks * 2 + (p.xs ? sum_bytes : 0)) * (uint32_t)S);
     const int per = NP + 1;  // copies per slice: the rows, then the sums
     for (int i = lane; i < S * per; i += 32) {
       const int sl = i / per, r = i - sl * per, slice = blockIdx.y * S + sl;
-      if (r < NP)
+      if (r < rows_used)
         bulk_copy_g2s(sAct + sl * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
                       &s_mbar);
-      else if (p.xs)
+      else if (r == NP && p.xs)
         bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
     }
   }
