@@ -448,7 +448,8 @@ def main():
         proj = "q4_umma_kernel" if os.environ.get("Q4D_GEMM_KERNEL") == "tcgen05" else "q4_span_kernel"
         head = "q4_umma_kernel" if os.environ.get("Q4D_GEMM_KERNEL") == "tcgen05" else "q4_round_kernel"
         class_kernel = {"gemm_qkv": proj, "gemm_o": proj, "gemm_gate_up": proj, "gemm_down": proj, "lm_head": head,
-                        "attention": "paged_attention_kernel", "moe_gate_up": "q4_gemm_kernel",
+                        "attention": ("paged_attention_t_kernel" if shape.n_q_heads // shape.n_kv_heads <= 8
+                                      else "paged_attention_kernel"), "moe_gate_up": "q4_gemm_kernel",
                         "moe_down": "q4_gemm_kernel", "rmsnorm": "rmsnorm_kernel", "embed": "embed_kernel",
                         "argmax": "argmax_finish_kernel", "moe_router": "moe_router_kernel"}
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel on the Llama-3.2-3B-shaped

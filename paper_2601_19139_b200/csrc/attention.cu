@@ -40,9 +40,11 @@ __device__ __forceinline__ void merge_head_chunk(const AttnArgs& p, int r, int a
   float den = 0.0f;
   if (valid) {
     float M = -INFINITY;
-#pragma unroll 8
+    // the merge runs in the last CTA of a request, after everything else: its loads go out in batches (16 maxima,
+    // then 8 chunks' partial results at a time) so that a request of a dozen chunks costs two round trips, not four
+#pragma unroll 16
     for (int c = 0; c < nc; ++c) M = fmaxf(M, __ldcg(p.part_ml + ((size_t)(s0 + c) * p.nq + a) * 2));
-#pragma unroll 4
+#pragma unroll 8
     for (int c = 0; c < nc; ++c) {
       const size_t qh = (size_t)(s0 + c) * p.nq + a;
       const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + qh * 2));
