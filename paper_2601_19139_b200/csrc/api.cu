@@ -130,13 +130,13 @@ Workspace carve(const q4d_shape& s, const MetaLayout& ml) {
   const int nqkv = (s.n_q_heads + 2 * s.n_kv_heads) * kHeadDim;
   const size_t qdim = (size_t)s.n_q_heads * kHeadDim;
   w.x = take(B * s.hidden * 2);
-  w.yp = take(B * s.hidden * 2);
+  w.yp = take(operand_elements(OPERAND_SLICED, s.hidden) * 2);  // the largest of the layouts
   w.ys = take((size_t)(s.hidden / 64) * 16 * 4);
   w.qkv = take(B * nqkv * 2);
   w.qbuf = take(B * qdim * 2);
-  w.ap = take(B * qdim * 2);
+  w.ap = take(operand_elements(OPERAND_SLICED, qdim) * 2);
   w.as = take((qdim / 64) * 16 * 4);
-  w.hp = take(B * (size_t)s.mlp_inter * 2 + 256);
+  w.hp = take(operand_elements(OPERAND_SLICED, s.mlp_inter) * 2 + 256);
   w.hs = take((size_t)(s.mlp_inter / 64) * 16 * 4 + 256);
   w.yplain = w.m_idx = w.m_wgt = w.m_ints = w.m_hp = w.m_hs = w.m_o = 0;
   if (s.n_experts) {
@@ -560,7 +560,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
   float* logits = logits_dev ? logits_dev : at<float>(m, m->lay.logits);
   const size_t layer_elems = (size_t)pool->num_blocks * nkv * kBlockSize * kHeadDim;
   const int qdim = nq * kHeadDim;
-  const int dense_layout = gemm_operand_layout(false);  // of the operands of the dense projections
+  const int dense_layout = gemm_operand_layout(false, n);  // of the operands of the dense projections
 
 #define Q4D_LAUNCH(cls, expr)                                                 \
   do {                                                                        \
@@ -628,7 +628,7 @@ int step_impl(q4d_model* m, q4d_kv_pool* pool, int32_t n, const int64_t* ids, co
       uint16_t* ehp = at<uint16_t>(m, m->lay.m_hp);
       float* ehs = at<float>(m, m->lay.m_hs);
       uint16_t* eo = at<uint16_t>(m, m->lay.m_o);
-      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, yplain, yp, ys, gemm_operand_layout(true), s));
+      Q4D_LAUNCH(Q4D_K_RMSNORM, launch_rmsnorm(x, lw.mlp_norm, sh.rms_eps, n, H, yplain, yp, ys, gemm_operand_layout(true, n), s));
       Q4D_LAUNCH(Q4D_K_MOE_ROUTER, launch_moe_router(mr, n, s));
       GemmArgs gu = gemm_args(m, lw.experts_gate_up, 2 * Ie, H, yp, ys, n, EPI_SILU_PACK, nullptr, 0);
       gu.out_xp = ehp, gu.out_xs = ehs;
@@ -1067,7 +1067,7 @@ constexpr size_t kOpAttnMeta = 1ull << 20;
 constexpr size_t kOpPartAcc = 64ull << 20;
 constexpr size_t kOpPartMl = 1ull << 20;
 constexpr int kOpMaxK = 32768;                         // widest operand the pack buffers hold
-constexpr size_t kOpPackXp = (size_t)16 * kOpMaxK * 2;  // fragment-ordered operand
+constexpr size_t kOpPackXp = (size_t)16 * kOpMaxK * 2 + kOpMaxK;  // fragment-ordered operand, with the sliced layout's padding
 constexpr size_t kOpPackXs = (size_t)(kOpMaxK / 64) * 16 * 4;
 constexpr size_t kOpPackOff = kOpCounters + kOpGemmPartial + kOpAttnMeta + kOpPartAcc + kOpPartMl;
 }  // namespace
@@ -1088,7 +1088,7 @@ int q4d_q4_gemm(const q4d_qtensor* w, int32_t N, int32_t K, const uint16_t* x, i
   uint16_t* xp = reinterpret_cast<uint16_t*>(sc + kOpPackOff);
   float* xs = reinterpret_cast<float*>(sc + kOpPackOff + kOpPackXp);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  cudaError_t e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false), st);
+  cudaError_t e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false, n), st);
   if (e != cudaSuccess) return fail_cuda(e, "q4_gemm (operand)");
   GemmArgs a;
   a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "kernels.h"
+
 namespace q4d {
 
 // ---- bf16 <-> f32 by bit pattern ------------------------------------------------
@@ -78,9 +80,17 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* 
 // {0,4,1,5,2,6,3,7} (so that a lane's 16 bytes are its B fragments of two k-steps), plus the fp32 sum of every
 // group of 64 elements, [K/64][16].  Producers build both with these helpers, always with the same summation
 // tree: ((e0+e1)+(e2+e3))+((e4+e5)+(e6+e7)) per chunk, then a pairwise tree over the 8 chunks of the group.
-// Element offset of chunk c (8 features) of request r in an operand of K features: layout 0 is [16][K], layout 1 is
-// [K/8][16][8] (all requests of a chunk side by side: the tensor-core kernel copies a K-range as one block).
+// Element offset of chunk c (8 features) of request r in an operand of K features.  Layout 0 is [16][K]; layout 1 is
+// [K/8][16][8] (all requests of a chunk side by side: the tensor-core kernel copies a K-range as one block); layout
+// 2 is [K/ks][16][ks + 8]: K cut into slices of ks features (operand_slice_features), the 16 rows of a slice side by
+// side, each followed by 8 unused elements -- byte for byte the shared-memory image the mma.sync kernels want (rows
+// 16 bytes apart modulo 128 for conflict-free fragment loads), so that a CTA stages a slice with ONE bulk copy: the
+// time to stage an operand is set by the number of copies, not by their bytes.
 __device__ __forceinline__ size_t operand_chunk_offset(int layout, int K, int r, int c) {
+  if (layout == 2) {
+    const int ks = operand_slice_features(K), k = c * 8, sl = k / ks;
+    return ((size_t)sl * 16 + r) * (ks + 8) + (k - sl * ks);
+  }
   return layout ? ((size_t)c * 16 + r) * 8 : (size_t)r * K + (size_t)c * 8;
 }
 __device__ __forceinline__ uint4 permute_chunk(const uint4 v) {

@@ -19,11 +19,23 @@ bool pdl_enabled();
 
 // ---- fragment-ordered GEMM operand ---------------------------------------------------
 // xp bf16 [16][K] (chunks of 8 permuted), xs f32 [K/64][16] (group sums); see common.cuh.
-// Two layouts of the bf16 elements exist: OPERAND_ROWS, [16][K] (the mma.sync kernels), and OPERAND_BLOCKED,
-// [K/8][16][8] (the tcgen05 kernel: a K-range of all requests is one contiguous block that the tensor core reads as
-// 8-request x 16-byte core matrices).  Both keep the order 0,4,1,5,2,6,3,7 inside a chunk of 8.
+// Three layouts of the bf16 elements exist: OPERAND_ROWS, [16][K] (the grouped projections of the MoE layers),
+// OPERAND_BLOCKED, [K/8][16][8] (the tcgen05 kernel: a K-range of all requests is one contiguous block that the
+// tensor core reads as 8-request x 16-byte core matrices), and OPERAND_SLICED, [K/ks][16][ks + 8] (the mma.sync
+// kernels of the dense projections: a slice of ks features of all requests is one contiguous block, already padded
+// like its shared-memory image).  All keep the order 0,4,1,5,2,6,3,7 inside a chunk of 8.
 enum GemmPrologue { PRO_PLAIN = 0, PRO_SILU_MUL = 1 };
-enum OperandLayout { OPERAND_ROWS = 0, OPERAND_BLOCKED = 1 };
+enum OperandLayout { OPERAND_ROWS = 0, OPERAND_BLOCKED = 1, OPERAND_SLICED = 2 };
+__host__ __device__ __forceinline__ int operand_slice_features(int K) {
+  const int quads = K >> 8;  // slices are the largest of 1024, 768, 512, 256 features that divides K
+  for (int c = 4; c > 1; --c)
+    if (quads % c == 0) return c << 8;
+  return 256;
+}
+__host__ __device__ __forceinline__ size_t operand_elements(int layout, int K) {  // elements an operand buffer needs
+  return layout == OPERAND_SLICED ? (size_t)(K / operand_slice_features(K)) * 16 * (operand_slice_features(K) + 8) : (size_t)16 * K;
+}
+
 cudaError_t launch_pack_operand(const uint16_t* x, int x_stride, int K, int n, int prologue, uint16_t* xp, float* xs,
                                 int layout, cudaStream_t s);
 
@@ -65,7 +77,7 @@ int gemm_counters_needed(int N);
 int gemm_row_blocks(int N, int K, int n, int epilogue);  // grid.x of the launch (size of argmax_partial)
 cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s);
 // The operand layout launch_q4_gemm expects for this call (grouped: the mixture-of-experts mode).
-int gemm_operand_layout(bool grouped);
+int gemm_operand_layout(bool grouped, int n);  // n: requests of the call
 
 // tcgen05 kernel (q4_umma.cu): tiles of 128 rows, K in `parts` across CTAs, stages of 256 features.
 struct UmmaPlan {

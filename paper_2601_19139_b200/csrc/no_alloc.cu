@@ -24,7 +24,8 @@ namespace {
 constexpr size_t kCounterBytes = 16 * 1024;          // 4096 row-tile counters
 constexpr size_t kPartialBytes = 8ull << 20;         // split-K partial sums
 constexpr int kMaxK = 16384;                         // widest input the operand buffers hold
-constexpr size_t kOperandBytes = (size_t)16 * kMaxK * 2 + (size_t)(kMaxK / 64) * 16 * 4;  // operand + group sums
+constexpr size_t kOperandXpBytes = (size_t)16 * kMaxK * 2 + kMaxK;  // operand rows with the padding of the sliced layout
+constexpr size_t kOperandBytes = kOperandXpBytes + (size_t)(kMaxK / 64) * 16 * 4;  // operand + group sums
 constexpr size_t kScratchBytes = kCounterBytes + kPartialBytes + kOperandBytes;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kScratchBytes];
@@ -83,8 +84,8 @@ extern "C" int q4d_q4_gemm_noalloc(const q4d_qtensor* w, int32_t N, int32_t K, c
   if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: clearing the counters failed");
   // the activations are first rearranged into the order the GEMM reads them in, inside the same array
   uint16_t* xp = reinterpret_cast<uint16_t*>(base + kCounterBytes + kPartialBytes);
-  float* xs = reinterpret_cast<float*>(base + kCounterBytes + kPartialBytes + (size_t)16 * kMaxK * 2);
-  e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false), s);
+  float* xs = reinterpret_cast<float*>(base + kCounterBytes + kPartialBytes + kOperandXpBytes);
+  e = launch_pack_operand(x, x_stride, K, n, prologue, xp, xs, gemm_operand_layout(false, n), s);
   if (e != cudaSuccess) return q4d_internal_fail(Q4D_ERR_CUDA, "q4_gemm_noalloc: operand rearrangement failed");
   GemmArgs a;
   a.qw = w->q, a.scales = w->scales, a.biases = w->biases, a.N = N, a.K = K, a.xp = xp, a.xs = xs, a.n = n;

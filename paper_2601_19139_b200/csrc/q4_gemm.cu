@@ -51,6 +51,7 @@ struct GemmParams {
   int ks;      // nominal K-slice (multiple of 256)
   int splits;  // gridDim.y
   int epilogue;
+  int out_ks, out_row_stride, out_slice_stride;  // out_xp: features per slice, elements between rows and between slices
   // grouped mode (MoE experts): blockIdx.z is a slot of the touched-expert list; the tensors of expert
   // expert_ids[slot] start expert_rows rows further per expert; operand and output move by their slot strides.
   const int* expert_ids;
@@ -380,7 +381,10 @@ __device__ __forceinline__ void tile_epilogue(const Params& p, const float (&acc
     const int col0 = tile * 8;
     if (lane < NP && lane < p.n && col0 < half_n) {
       const uint4 v = *reinterpret_cast<const uint4*>(sH + lane * 8);
-      *reinterpret_cast<uint4*>(p.out_xp + (size_t)lane * half_n + col0) = permute_chunk(v);
+      // element (lane, col0) of the consumer's operand: slices of out_ks features, strides set by the host
+      const int sl = col0 / p.out_ks;
+      *reinterpret_cast<uint4*>(p.out_xp + (size_t)sl * p.out_slice_stride + (size_t)lane * p.out_row_stride +
+                                (col0 - sl * p.out_ks)) = permute_chunk(v);
     }
     __syncwarp();
     return;
@@ -471,6 +475,8 @@ struct RoundParams {
   float* partial;          // [parts][T][MT * 16 * 8 NT] sums of a tile over one part of K (parts > 1 only)
   int* counters;           // [T], zero between launches (parts > 1 only)
   int N, K, n, out_stride, epilogue;
+  int out_ks, out_row_stride, out_slice_stride;  // out_xp: features per slice, elements between rows and between slices
+  int xp_layout;   // layout of xp: OPERAND_SLICED (one copy per slice) or OPERAND_ROWS (one copy per row and slice)
   int T;   // row tiles of MT sub-tiles
   int Tsub;  // sub-tiles of 16 rows (SiLU epilogue: 8 gate rows and the 8 matching up rows)
   int Q;   // stages per K-slice
@@ -512,7 +518,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   return false;
 }
 
-template <int NT, int STAGES>
+template <int NT, int STAGES, bool SLICED>  // SLICED: the operand's layout (one copy per slice) or plain rows
 __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundParams p) {
   constexpr int NP = 8 * NT, MT = kRoundMT, RW = kRoundRows;
   constexpr int kEs = NP + 1;
@@ -600,12 +606,16 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
   // Only the rows of requests that exist are fetched; the other columns of the MMAs multiply whatever the buffer
   // holds and their results are never stored.
   const int rows_used = p.n < NP ? p.n : NP;
-  const uint32_t slice_bytes = (uint32_t)(rows_used * ks * 2 + (p.xs ? sum_bytes : 0));
+  constexpr bool sliced = SLICED;  // a sliced row comes with its padding
+  const uint32_t slice_bytes = (uint32_t)(rows_used * (sliced ? b_stride : ks * 2) + (p.xs ? sum_bytes : 0));
   auto stage_acts = [&](int gstep) {  // the lanes of warp 0 issue the copies side by side
     if (warp == 0) {
       const int buf = gstep & 1, slice = blockIdx.y * S + gstep % S;
       if (lane == 0) mbar_expect_tx(&s_mbar[buf], slice_bytes);
-      if (lane < rows_used)
+      if (sliced && lane == 0)  // the slice's rows are one contiguous block, padded like their image here
+        bulk_copy_g2s(sAct + buf * act_bytes, p.xp + (size_t)slice * 16 * (ks + 8), (uint32_t)(rows_used * b_stride),
+                      &s_mbar[buf]);
+      else if (!sliced && lane < rows_used)
         bulk_copy_g2s(sAct + buf * act_bytes + lane * b_stride, p.xp + (size_t)lane * p.K + (size_t)slice * ks,
                       (uint32_t)(ks * 2), &s_mbar[buf]);
       else if (lane == NP && p.xs)
@@ -896,7 +906,7 @@ __device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, co
   }
 }
 
-template <int NT, int STAGES>
+template <int NT, int STAGES, bool SLICED>  // SLICED: the operand's layout (one copy per slice) or plain rows
 __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundParams p) {
   static_assert(kRoundMT == 1, "the span kernel works on 16-row tiles");
   constexpr int NP = 8 * NT, W = kRoundWarps;
@@ -959,15 +969,22 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
     // only the rows of requests that exist are fetched: the other columns of the MMAs multiply whatever the buffer
     // holds and their results are never stored
     const int rows_used = p.n < NP ? p.n : NP;
-    if (lane == 0) mbar_expect_tx(&s_mbar, (uint32_t)(rows_used * ks * 2 + (p.xs ? sum_bytes : 0)) * (uint32_t)S);
-    const int per = NP + 1;  // copies per slice: the rows, then the sums
+    const int row_bytes = SLICED ? b_stride : ks * 2;  // a sliced row comes with its padding
+    if (lane == 0) mbar_expect_tx(&s_mbar, (uint32_t)(rows_used * row_bytes + (p.xs ? sum_bytes : 0)) * (uint32_t)S);
+    // a slice of the operand is one contiguous block in global memory, padded like its image here: one copy each
+    // for the rows and for the sums (the copy engine's time goes with the number of copies, not with their bytes)
+    const int per = NP + 1;  // copies per slice at most: the rows, then the sums
     for (int i = lane; i < S * per; i += 32) {
       const int sl = i / per, r = i - sl * per, slice = blockIdx.y * S + sl;
-      if (r < rows_used)
+      if (r == NP) {
+        if (p.xs) bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
+      } else if (SLICED) {
+        if (r == 0)
+          bulk_copy_g2s(sAct + sl * act_bytes, p.xp + (size_t)slice * 16 * (ks + 8), (uint32_t)(rows_used * b_stride), &s_mbar);
+      } else if (r < rows_used) {
         bulk_copy_g2s(sAct + sl * act_bytes + r * b_stride, p.xp + (size_t)r * p.K + (size_t)slice * ks, (uint32_t)(ks * 2),
                       &s_mbar);
-      else if (r == NP && p.xs)
-        bulk_copy_g2s(sSum + sl * (sum_bytes / 4), p.xs + (size_t)slice * Q * 4 * 16, (uint32_t)sum_bytes, &s_mbar);
+      }
     }
   }
   __syncwarp();  // lanes that have nothing to issue go on to poll the mbarrier: they must not starve the others
@@ -1121,12 +1138,8 @@ RoundPlan plan_rounds(int N, int K, int n, int epilogue, int sm_count) {
   t.nt = n <= 8 ? 1 : 2;
   t.stages = t.nt == 1 ? 3 : 2;  // ring slots per warp; deeper rings measured slower (LM head: 4 -> 142 us, 5 -> 171 us, 2 -> 137 us)
   const int quads = K / 256;
-  t.Q = 1;
-  for (int c = kMaxQuadsPerSlice; c >= 1; --c)
-    if (quads % c == 0) {
-      t.Q = c;
-      break;
-    }
+  static_assert(kMaxQuadsPerSlice == 4, "operand_slice_features cuts K into slices of at most 4 x 256 features");
+  t.Q = operand_slice_features(K) / 256;  // the producers lay the operand out in these slices
   const int slices = quads / t.Q;
   // A CTA re-reads the activations of its part of K for every round, so K is cut into parts of at most four
   // slices: beyond that the activations would outweigh the CTA's weights.
@@ -1262,9 +1275,13 @@ int gemm_row_blocks(int N, int K, int n, int epilogue) {
   return t.ctas * t.parts * kRoundWarps;  // one argmax partial per warp of the grid
 }
 
-int gemm_operand_layout(bool grouped) {
+int gemm_operand_layout(bool grouped, int n) {
   (void)sm_count_or_default();
-  return (grouped || g_legacy) ? OPERAND_ROWS : OPERAND_BLOCKED;
+  if (grouped) return OPERAND_ROWS;
+  if (!g_legacy) return OPERAND_BLOCKED;
+  // One or two requests: a slice is one or two row copies either way, and plain rows measured faster there
+  // (8B-shaped batch 1: 2.76 against 2.84 ms per step); from three requests on one copy per slice wins.
+  return n <= 2 ? OPERAND_ROWS : OPERAND_SLICED;
 }
 
 cudaError_t gemm_init() {
@@ -1281,12 +1298,11 @@ cudaError_t gemm_init() {
     e = cudaFuncSetAttribute(q4_gemm_kernel<2, 2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(q4_gemm_kernel<1, 2, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<1, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(q4_round_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(q4_span_kernel<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  auto big_smem = [&](auto kernel) {
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big);
+  };
+  big_smem(q4_round_kernel<1, 3, true>), big_smem(q4_round_kernel<1, 3, false>), big_smem(q4_round_kernel<2, 2, true>);
+  big_smem(q4_span_kernel<1, 2, true>), big_smem(q4_span_kernel<1, 2, false>), big_smem(q4_span_kernel<2, 2, true>);
   if (e != cudaSuccess) return e;
   if (const char* f = getenv("Q4D_GEMM_KERNEL")) g_legacy = strcmp(f, "tcgen05") != 0;
   g_sm_count = sms;
@@ -1310,6 +1326,12 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     p.qw = a.qw, p.scales = a.scales, p.biases = a.biases, p.xp = a.xp, p.xs = a.xs, p.out = a.out;
     p.out_xp = a.out_xp, p.argmax_partial = a.argmax_partial, p.status = a.status;
     p.N = a.N, p.K = a.K, p.n = a.n, p.out_stride = a.out_stride, p.epilogue = a.epilogue;
+    p.xp_layout = gemm_operand_layout(false, a.n);
+    {  // the SiLU epilogue feeds a dense projection of N / 2 input features in the same layout
+      const int k2 = a.N / 2, ks2 = p.xp_layout == OPERAND_SLICED && k2 % 256 == 0 ? operand_slice_features(k2) : k2;
+      const bool sl2 = p.xp_layout == OPERAND_SLICED && k2 % 256 == 0;
+      p.out_ks = ks2, p.out_row_stride = sl2 ? ks2 + 8 : k2, p.out_slice_stride = sl2 ? 16 * (ks2 + 8) : 0;
+    }
     p.T = t.T, p.Tsub = t.Tsub, p.Q = t.Q, p.S = t.S, p.kw = t.kw;
     p.partial = a.partial, p.counters = a.counters;
     if (t.parts > 1 && (!a.partial || !a.counters || t.partial_bytes > a.partial_bytes || t.T > a.counters_len))
@@ -1317,12 +1339,16 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
     const int elem = a.epilogue == EPI_F32 ? 4 : 2;
     p.vec_ok = a.out && (reinterpret_cast<uintptr_t>(a.out) % 16 == 0) && ((size_t)a.out_stride * elem % 16 == 0);
     const dim3 grid(t.ctas, t.parts), block(kRoundThreads);
+    const bool sliced = p.xp_layout == OPERAND_SLICED;
+    if (t.nt == 2 && !sliced) return cudaErrorInvalidValue;  // more than eight requests always come sliced
     if (t.span) {
-      if (t.nt == 1) return launch_kernel(q4_span_kernel<1, 2>, grid, block, t.span_smem, s, p);
-      return launch_kernel(q4_span_kernel<2, 2>, grid, block, t.span_smem, s, p);
+      if (t.nt == 2) return launch_kernel(q4_span_kernel<2, 2, true>, grid, block, t.span_smem, s, p);
+      if (sliced) return launch_kernel(q4_span_kernel<1, 2, true>, grid, block, t.span_smem, s, p);
+      return launch_kernel(q4_span_kernel<1, 2, false>, grid, block, t.span_smem, s, p);
     }
-    if (t.nt == 1) return launch_kernel(q4_round_kernel<1, 3>, grid, block, t.smem, s, p);
-    return launch_kernel(q4_round_kernel<2, 2>, grid, block, t.smem, s, p);
+    if (t.nt == 2) return launch_kernel(q4_round_kernel<2, 2, true>, grid, block, t.smem, s, p);
+    if (sliced) return launch_kernel(q4_round_kernel<1, 3, true>, grid, block, t.smem, s, p);
+    return launch_kernel(q4_round_kernel<1, 3, false>, grid, block, t.smem, s, p);
   }
   const Tiling t = choose_tiling(a.N, a.K, a.n, a.epilogue, g_sm_count, grouped);
   GemmParams p;
@@ -1334,6 +1360,7 @@ cudaError_t launch_q4_gemm(const GemmArgs& a, cudaStream_t s) {
   p.partial = a.partial, p.counters = a.counters;
   p.N = a.N, p.K = a.K, p.n = a.n, p.out_stride = a.out_stride;
   p.ks = t.qps * 256, p.splits = t.splits, p.epilogue = a.epilogue;
+  p.out_ks = a.N / 2 > 0 ? a.N / 2 : 1, p.out_row_stride = a.N / 2, p.out_slice_stride = 0;  // plain rows
   if (t.splits > 1) {
     if (!a.partial || !a.counters || tiling_partial_bytes(t) > a.partial_bytes || t.rowblocks > a.counters_len)
       return cudaErrorInvalidValue;
