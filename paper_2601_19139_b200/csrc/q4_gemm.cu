@@ -1065,9 +1065,12 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
       for (int c = 0; c < 4; ++c) acc[nt][c] = 0.0f;
+    const int tile_first = tl * SQ;  // the tile's first stage
+#pragma unroll 4
     for (int w2 = span; w2 <= last; ++w2) {
-      if (span_begin(w2 + 1) == span_begin(w2)) continue;   // an empty span (fewer stages than warps)
-      const int sel = (span_begin(w2) / SQ == tl) ? 0 : 1;  // the tile is that span's first or second
+      const int b0 = span_begin(w2);
+      if (span_begin(w2 + 1) == b0) continue;  // an empty span (fewer stages than warps)
+      const int sel = b0 < tile_first ? 1 : 0;  // the tile is that span's first tile, or its second
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
         const float4 v = sP[((w2 * 2 + sel) * NT + nt) * 32 + lane];
