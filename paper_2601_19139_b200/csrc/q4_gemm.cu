@@ -834,27 +834,6 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
 // tail of one tile and the head of the next at most, and each warp refills the ring slot it has just multiplied.
 // At the end the warps leave their (one or two) partial sums in shared memory, and the warp that holds a tile's first
 // stage adds the tile's partial sums in warp order and applies the epilogue.
-__device__ __forceinline__ void span_issue_stage(const RoundParams& p, unsigned char* stg, int sub, int stage_k, bool silu,
-                                                 int half_n, int lane) {
-  auto row_of = [&](int r) -> int {
-    if (!silu) return min(sub * 16 + r, p.N - 1);
-    return r < 8 ? min(sub * 8 + r, half_n - 1) : min(half_n + sub * 8 + (r - 8), p.N - 1);
-  };
-  const int kq = stage_k * 256;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = i * 4 + (lane >> 3);
-    const unsigned char* src =
-        reinterpret_cast<const unsigned char*>(p.qw + (size_t)row_of(r) * (p.K >> 3) + (kq >> 3)) + (lane & 7) * 16;
-    cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), src);
-  }
-  if (lane < 16) {
-    const size_t off = (size_t)row_of(lane) * (p.K >> 6) + (kq >> 6);
-    cp_async8(stg + 16 * 128 + lane * kSbBytes, p.scales + off);
-    cp_async8(stg + 16 * 128 + lane * kSbBytes + 8, p.biases + off);
-  }
-}
-
 // acc += the stage's 16 rows x 256 input features against the staged operand (sB: the slice, sX: its group sums,
 // cq: the stage's place in the slice).
 template <int NT>
@@ -944,13 +923,45 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
     else tl = tlA + 1, j = i - lenA;
   };
 
+  const int q_recip = (65536 + Q - 1) / Q;  // j / Q == (j * q_recip) >> 16 for j < 4096 and Q <= 4
+  // The addresses of a tile's rows are worked out once per tile (a span touches two tiles at most), not per stage:
+  // a stage then costs five additions instead of five 64-bit multiplications with their row clamps.
+  const unsigned char* row_src[4];  // rows 4i + lane / 8 of the tile, at this lane's 16 bytes of feature 0
+  size_t sb_off = 0;                // row `lane` of the tile in the scale / bias tensors (lanes < 16)
+  int rows_tl = -1;
+  auto issue_stage = [&](unsigned char* stg, int tl, int j) {
+    if (tl != rows_tl) {
+      rows_tl = tl;
+      const int sub = t0 + tl;
+      auto row_of = [&](int r) -> int {
+        if (!silu) return min(sub * 16 + r, p.N - 1);
+        return r < 8 ? min(sub * 8 + r, half_n - 1) : min(half_n + sub * 8 + (r - 8), p.N - 1);
+      };
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        row_src[i] = reinterpret_cast<const unsigned char*>(p.qw + (size_t)row_of(i * 4 + (lane >> 3)) * (p.K >> 3)) +
+                     (lane & 7) * 16;
+      sb_off = (size_t)row_of(lane & 15) * (p.K >> 6);
+    }
+    const int kq = (part_j0 + j) * 256;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int r = i * 4 + (lane >> 3);
+      cp_async16(stg + r * 128 + (((lane & 7) ^ (r & 7)) << 4), row_src[i] + (kq >> 1));
+    }
+    if (lane < 16) {
+      cp_async8(stg + 16 * 128 + lane * kSbBytes, p.scales + sb_off + (kq >> 6));
+      cp_async8(stg + 16 * 128 + lane * kSbBytes + 8, p.biases + sb_off + (kq >> 6));
+    }
+  };
+
   // Weights do not depend on the preceding kernel: fill the ring before waiting for it.
 #pragma unroll
   for (int i = 0; i < STAGES; ++i) {
     if (i < cnt) {
       int tl, j;
       stage_of(i, tl, j);
-      span_issue_stage(p, ring + i * kRoundStage, t0 + tl, part_j0 + j, silu, half_n, lane);
+      issue_stage(ring + i * kRoundStage, tl, j);
     }
     cp_async_commit();
   }
@@ -1024,14 +1035,14 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
 #pragma unroll
         for (int c = 0; c < 4; ++c) first[nt][c] = acc[nt][c], acc[nt][c] = 0.0f;
     }
-    const int sl = j / Q, cq = j - sl * Q;
+    const int sl = (j * q_recip) >> 16, cq = j - sl * Q;  // j / Q for the few stages of a tile
     span_multiply_stage<NT>(ring + slot * kRoundStage, sAct + sl * act_bytes, sSum + sl * (sum_bytes / 4), b_stride, cq, g, t,
                             acc);
     __syncwarp();
     if (i + STAGES < cnt) {  // refill the slot just multiplied
       int tl2, j2;
       stage_of(i + STAGES, tl2, j2);
-      span_issue_stage(p, ring + slot * kRoundStage, t0 + tl2, part_j0 + j2, silu, half_n, lane);
+      issue_stage(ring + slot * kRoundStage, tl2, j2);
     }
     cp_async_commit();
     if (++slot == STAGES) slot = 0;
