@@ -76,6 +76,19 @@ __device__ __forceinline__ void unpack_word(uint32_t w, uint32_t (&p)[4]) {
   p[3] = and_or(w >> 9, kMask, kSixteen);
 }
 
+// two fp32 FMAs in one instruction: c = a * b + c on both halves, each rounded like a scalar FMA
+__device__ __forceinline__ void fma_f32x2(unsigned long long& c, unsigned long long a, unsigned long long b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(c) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
 __device__ __forceinline__ float bf16_at(const uint2& v, int i) {
   uint32_t w = (i >> 1) ? v.y : v.x;
   return (i & 1) ? bf16_hi(w) : bf16_lo(w);
@@ -870,6 +883,8 @@ __device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, co
     // sum (16 + q) x = 16 X + sum q x, so the bias that multiplies X becomes b - 16 s
     const float s_lo = bf16_at(sc[0], gi), s_hi = bf16_at(sc[1], gi);
     const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[1], gi));
+    const unsigned long long s_lo2 = pack_f32x2(s_lo, s_lo), s_hi2 = pack_f32x2(s_hi, s_hi);
+    const unsigned long long b_lo2 = pack_f32x2(b_lo, b_lo), b_hi2 = pack_f32x2(b_hi, b_hi);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       float pc[4];
@@ -877,10 +892,15 @@ __device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, co
       mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
       mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
       mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
-      acc[nt][0] = fmaf(s_lo, pc[0], fmaf(b_lo, xs[nt].x, acc[nt][0]));
-      acc[nt][1] = fmaf(s_lo, pc[1], fmaf(b_lo, xs[nt].y, acc[nt][1]));
-      acc[nt][2] = fmaf(s_hi, pc[2], fmaf(b_hi, xs[nt].x, acc[nt][2]));
-      acc[nt][3] = fmaf(s_hi, pc[3], fmaf(b_hi, xs[nt].y, acc[nt][3]));
+      // acc = s * pc + (b * xs + acc), two requests per packed instruction (each half rounds like a scalar FMA)
+      const unsigned long long x2 = pack_f32x2(xs[nt].x, xs[nt].y);
+      unsigned long long a01 = pack_f32x2(acc[nt][0], acc[nt][1]), a23 = pack_f32x2(acc[nt][2], acc[nt][3]);
+      fma_f32x2(a01, b_lo2, x2);
+      fma_f32x2(a23, b_hi2, x2);
+      fma_f32x2(a01, s_lo2, pack_f32x2(pc[0], pc[1]));
+      fma_f32x2(a23, s_hi2, pack_f32x2(pc[2], pc[3]));
+      unpack_f32x2(a01, acc[nt][0], acc[nt][1]);
+      unpack_f32x2(a23, acc[nt][2], acc[nt][3]);
     }
   }
 }
