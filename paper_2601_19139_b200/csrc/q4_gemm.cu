@@ -89,6 +89,20 @@ __device__ __forceinline__ void unpack_f32x2(unsigned long long v, float& lo, fl
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
 }
 
+// acc += s * pc + b * xs for the 2 x 2 block of an MMA fragment (rows g, g + 8; requests 2t, 2t + 1): s and b per row,
+// xs per request; two requests per packed instruction, each half rounded like the scalar fmaf(s, pc, fmaf(b, xs, acc)).
+__device__ __forceinline__ void scale_bias_fma(float (&acc)[4], const float (&pc)[4], float s_lo, float s_hi, float b_lo,
+                                               float b_hi, float2 xs) {
+  const unsigned long long x2 = pack_f32x2(xs.x, xs.y);
+  unsigned long long a01 = pack_f32x2(acc[0], acc[1]), a23 = pack_f32x2(acc[2], acc[3]);
+  fma_f32x2(a01, pack_f32x2(b_lo, b_lo), x2);
+  fma_f32x2(a23, pack_f32x2(b_hi, b_hi), x2);
+  fma_f32x2(a01, pack_f32x2(s_lo, s_lo), pack_f32x2(pc[0], pc[1]));
+  fma_f32x2(a23, pack_f32x2(s_hi, s_hi), pack_f32x2(pc[2], pc[3]));
+  unpack_f32x2(a01, acc[0], acc[1]);
+  unpack_f32x2(a23, acc[2], acc[3]);
+}
+
 __device__ __forceinline__ float bf16_at(const uint2& v, int i) {
   uint32_t w = (i >> 1) ? v.y : v.x;
   return (i & 1) ? bf16_hi(w) : bf16_lo(w);
@@ -257,10 +271,7 @@ __global__ void __launch_bounds__(kThreads, (MT == 1) ? 2 : 1) q4_gemm_kernel(co
           mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
           mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
           mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
-          acc[mt][nt][0] = fmaf(s_lo, pc[0], fmaf(b_lo, xs[nt].x, acc[mt][nt][0]));
-          acc[mt][nt][1] = fmaf(s_lo, pc[1], fmaf(b_lo, xs[nt].y, acc[mt][nt][1]));
-          acc[mt][nt][2] = fmaf(s_hi, pc[2], fmaf(b_hi, xs[nt].x, acc[mt][nt][2]));
-          acc[mt][nt][3] = fmaf(s_hi, pc[3], fmaf(b_hi, xs[nt].y, acc[mt][nt][3]));
+          scale_bias_fma(acc[mt][nt], pc, s_lo, s_hi, b_lo, b_hi, xs[nt]);
         }
       }
     }
@@ -729,10 +740,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
               mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
               mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
               mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
-              acc[mt][nt][0] = fmaf(s_lo, pc[0], fmaf(b_lo, xs[nt].x, acc[mt][nt][0]));
-              acc[mt][nt][1] = fmaf(s_lo, pc[1], fmaf(b_lo, xs[nt].y, acc[mt][nt][1]));
-              acc[mt][nt][2] = fmaf(s_hi, pc[2], fmaf(b_hi, xs[nt].x, acc[mt][nt][2]));
-              acc[mt][nt][3] = fmaf(s_hi, pc[3], fmaf(b_hi, xs[nt].y, acc[mt][nt][3]));
+              scale_bias_fma(acc[mt][nt], pc, s_lo, s_hi, b_lo, b_hi, xs[nt]);
             }
           }
         }
@@ -883,8 +891,6 @@ __device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, co
     // sum (16 + q) x = 16 X + sum q x, so the bias that multiplies X becomes b - 16 s
     const float s_lo = bf16_at(sc[0], gi), s_hi = bf16_at(sc[1], gi);
     const float b_lo = fmaf(-16.0f, s_lo, bf16_at(bi[0], gi)), b_hi = fmaf(-16.0f, s_hi, bf16_at(bi[1], gi));
-    const unsigned long long s_lo2 = pack_f32x2(s_lo, s_lo), s_hi2 = pack_f32x2(s_hi, s_hi);
-    const unsigned long long b_lo2 = pack_f32x2(b_lo, b_lo), b_hi2 = pack_f32x2(b_hi, b_hi);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       float pc[4];
@@ -892,15 +898,7 @@ __device__ __forceinline__ void span_multiply_stage(const unsigned char* stg, co
       mma_bf16(pc, l0[2], h0[2], l0[3], h0[3], bf[nt][0].z, bf[nt][0].w);
       mma_bf16(pc, l1[0], h1[0], l1[1], h1[1], bf[nt][1].x, bf[nt][1].y);
       mma_bf16(pc, l1[2], h1[2], l1[3], h1[3], bf[nt][1].z, bf[nt][1].w);
-      // acc = s * pc + (b * xs + acc), two requests per packed instruction (each half rounds like a scalar FMA)
-      const unsigned long long x2 = pack_f32x2(xs[nt].x, xs[nt].y);
-      unsigned long long a01 = pack_f32x2(acc[nt][0], acc[nt][1]), a23 = pack_f32x2(acc[nt][2], acc[nt][3]);
-      fma_f32x2(a01, b_lo2, x2);
-      fma_f32x2(a23, b_hi2, x2);
-      fma_f32x2(a01, s_lo2, pack_f32x2(pc[0], pc[1]));
-      fma_f32x2(a23, s_hi2, pack_f32x2(pc[2], pc[3]));
-      unpack_f32x2(a01, acc[nt][0], acc[nt][1]);
-      unpack_f32x2(a23, acc[nt][2], acc[nt][3]);
+      scale_bias_fma(acc[nt], pc, s_lo, s_hi, b_lo, b_hi, xs[nt]);
     }
   }
 }
