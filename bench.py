@@ -455,7 +455,7 @@ def main():
         # DRAM bytes per algorithmic byte from one `ncu --set full` capture of each kernel (see profiles/: the span kernel
         # on a gate/up-shaped projection alone, attention on the Llama-3.2-3B-shaped batch-16 case); traffic is
         # proportional to the bytes streamed, so it is scaled to this launch.
-        traffic_ratio = {"q4_span_kernel": 1.006, "paged_attention_t_kernel": 1.037}
+        traffic_ratio = {"q4_span_kernel": 1.005, "paged_attention_t_kernel": 1.037}
         total_prof_ms = sum(v[0] for v in prof.values())
         classes = {k: {"ms_per_step": v[0] / args.profile_steps, "launches_per_step": v[1] / args.profile_steps,
                        "share": v[0] / total_prof_ms, "kernel": class_kernel.get(k, k)} for k, v in prof.items() if v[1]}
