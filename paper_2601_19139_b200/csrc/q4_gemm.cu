@@ -626,7 +626,8 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_round_kernel(const RoundP
 
   grid_dependency_wait();
 
-  // One bulk copy per request row of the slice (and one for its group sums), tracked by the buffer's mbarrier.
+  // A slice arrives as one bulk copy of all its rows (sliced layout) or one per request row (plain rows), plus one
+  // for its group sums, tracked by the buffer's mbarrier.
   // Only the rows of requests that exist are fetched; the other columns of the MMAs multiply whatever the buffer
   // holds and their results are never stored.
   const int rows_used = p.n < NP ? p.n : NP;
@@ -992,8 +993,8 @@ __global__ void __launch_bounds__(kRoundThreads, 1) q4_span_kernel(const RoundPa
 
   grid_dependency_wait();
 
-  // every slice of the operand (and its group sums): one bulk copy per request row, all on one mbarrier, issued by
-  // the lanes of warp 0 side by side (a single thread would spend microseconds issuing up to 68 copies)
+  // every slice of the operand (and its group sums) on one mbarrier: one bulk copy per slice in the sliced layout,
+  // one per request row and slice with plain rows, issued by the lanes of warp 0 side by side
   if (warp == 0) {
     // only the rows of requests that exist are fetched: the other columns of the MMAs multiply whatever the buffer
     // holds and their results are never stored
